@@ -1,0 +1,178 @@
+"""numpy front end of the C oracle (``ref_gemm.c``) -- TEST INFRASTRUCTURE, not the product.
+
+Matrices are passed the way BLAS sees them: a flat numpy array holding column-major storage
+plus a leading dimension, X(r, c) = X[r + c*ldx].  Real arrays are float64 or float32; complex
+arrays are complex128 (interleaved re, im; leading dimensions in complex elements).
+
+  ref_gemm      the definition in working precision (Section 2.1 sum of rank-1 updates with the
+                BLAS alpha/beta/op/ld semantics); updates C in place.
+  ref_gemm_hi   the same sum accumulated in a wider type, plus the magnitude sum S used by
+                forward error bounds; returns (C_hi, S) and leaves C untouched.
+  ref_zgemm_4m  complex GEMM assembled from four calls of the real oracle on split planes (the
+                4M formulation), used to check that formulation against direct complex arithmetic.
+"""
+from __future__ import annotations
+
+import ctypes
+from ctypes import c_char, c_double, c_float, c_int, c_int64, c_void_p
+
+import numpy as np
+
+from . import build as _build
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(str(_build.build()))
+        real_tail = [c_char, c_char, c_int64, c_int64, c_int64]
+        _lib.ref_dgemm.argtypes = real_tail + [c_double, c_void_p, c_int64, c_void_p, c_int64, c_double, c_void_p,
+                                               c_int64, c_void_p, c_int64]
+        _lib.ref_sgemm.argtypes = real_tail + [c_float, c_void_p, c_int64, c_void_p, c_int64, c_float, c_void_p,
+                                               c_int64, c_void_p, c_int64]
+        _lib.ref_dgemm_hi.argtypes = real_tail + [c_double, c_void_p, c_int64, c_void_p, c_int64, c_double, c_void_p,
+                                                  c_int64, c_void_p, c_void_p, c_int64, c_void_p, c_int64]
+        _lib.ref_sgemm_hi.argtypes = real_tail + [c_float, c_void_p, c_int64, c_void_p, c_int64, c_float, c_void_p,
+                                                  c_int64, c_void_p, c_void_p, c_int64, c_void_p, c_int64]
+        _lib.ref_zgemm.argtypes = real_tail + [c_void_p, c_void_p, c_int64, c_void_p, c_int64, c_void_p, c_void_p,
+                                               c_int64, c_void_p, c_int64]
+        _lib.ref_zgemm_hi.argtypes = real_tail + [c_void_p, c_void_p, c_int64, c_void_p, c_int64, c_void_p, c_void_p,
+                                                  c_int64, c_void_p, c_void_p, c_int64, c_void_p, c_int64]
+        for fn in ("ref_dgemm", "ref_sgemm", "ref_dgemm_hi", "ref_sgemm_hi", "ref_zgemm", "ref_zgemm_hi",
+                   "ref_num_threads"):
+            getattr(_lib, fn).restype = c_int
+    return _lib
+
+
+def num_threads() -> int:
+    """OpenMP threads the oracle uses."""
+    return lib().ref_num_threads()
+
+
+def _tr(c: str) -> bytes:
+    return c.encode("ascii")[:1]
+
+
+def _flat(x: np.ndarray, dtype) -> np.ndarray:
+    if not isinstance(x, np.ndarray) or x.dtype != dtype or x.ndim != 1 or not x.flags.c_contiguous:
+        raise TypeError(f"expected a flat contiguous numpy array of {dtype}")
+    return x
+
+
+def _need(x: np.ndarray, ld: int, ncols: int, nrows: int, what: str) -> None:
+    if ncols > 0 and nrows > 0 and x.size < ld * (ncols - 1) + nrows:
+        raise ValueError(f"{what}: storage of {x.size} elements is too small for ld={ld}, {nrows}x{ncols}")
+
+
+def _cols(cols):
+    if cols is None:
+        return None, 0, None
+    arr = np.ascontiguousarray(np.asarray(cols, dtype=np.int64))
+    return arr.ctypes.data, arr.size, arr
+
+
+def _check_storage(transa, transb, m, n, k, A, lda, B, ldb, C, ldc, read_ab):
+    ta, tb = transa in "TtCc", transb in "TtCc"
+    if read_ab:
+        _need(A, lda, m if ta else k, k if ta else m, "A")
+        _need(B, ldb, k if tb else n, n if tb else k, "B")
+    _need(C, ldc, n, m, "C")
+
+
+def ref_gemm(transa, transb, m, n, k, alpha, A, lda, B, ldb, beta, C, ldc, cols=None) -> None:
+    """C := alpha*op(A)*op(B) + beta*C by the plain definition; C (flat storage) is updated in place."""
+    dt = C.dtype
+    if dt == np.complex128:
+        al = np.array([complex(alpha).real, complex(alpha).imag], dtype=np.float64)
+        be = np.array([complex(beta).real, complex(beta).imag], dtype=np.float64)
+        fn, args_a, args_b = lib().ref_zgemm, al.ctypes.data, be.ctypes.data
+        read_ab = not (al[0] == 0 and al[1] == 0) and k > 0
+    elif dt == np.float64:
+        fn, args_a, args_b = lib().ref_dgemm, float(alpha), float(beta)
+        read_ab = alpha != 0 and k > 0
+    elif dt == np.float32:
+        fn, args_a, args_b = lib().ref_sgemm, float(np.float32(alpha)), float(np.float32(beta))
+        read_ab = np.float32(alpha) != 0 and k > 0
+    else:
+        raise TypeError(f"unsupported dtype {dt}")
+    _flat(A, dt), _flat(B, dt), _flat(C, dt)
+    cptr, ncols, keep = _cols(cols)
+    rc = fn(_tr(transa), _tr(transb), m, n, k, args_a, A.ctypes.data, lda, B.ctypes.data, ldb, args_b, C.ctypes.data,
+            ldc, cptr, ncols)
+    if rc != 0:
+        raise ValueError(f"oracle rejected argument {-rc}")
+    if m > 0 and n > 0:
+        _check_storage(transa, transb, m, n, k, A, lda, B, ldb, C, ldc, read_ab)
+    del keep
+
+
+def ref_gemm_hi(transa, transb, m, n, k, alpha, A, lda, B, ldb, beta, C, ldc, cols=None):
+    """Wide-accumulation result and magnitude sum S; returns (C_hi, S) as flat arrays with leading dimension m.
+
+    For complex data C_hi is complex128 and S holds one bound term per element (valid for both components).
+    Columns outside `cols` are left as NaN.
+    """
+    dt = C.dtype
+    _flat(A, dt), _flat(B, dt), _flat(C, dt)
+    ldo = max(1, m)
+    Chi = np.full(ldo * max(n, 1), np.nan, dtype=dt)
+    S = np.full(ldo * max(n, 1), np.nan, dtype=np.float64)
+    cptr, ncols, keep = _cols(cols)
+    if m > 0 and n > 0:
+        _check_storage(transa, transb, m, n, k, A, lda, B, ldb, C, ldc, True)
+    if dt == np.complex128:
+        al = np.array([complex(alpha).real, complex(alpha).imag], dtype=np.float64)
+        be = np.array([complex(beta).real, complex(beta).imag], dtype=np.float64)
+        rc = lib().ref_zgemm_hi(_tr(transa), _tr(transb), m, n, k, al.ctypes.data, A.ctypes.data, lda, B.ctypes.data,
+                                ldb, be.ctypes.data, C.ctypes.data, ldc, Chi.ctypes.data, S.ctypes.data, ldo, cptr,
+                                ncols)
+    elif dt == np.float64:
+        rc = lib().ref_dgemm_hi(_tr(transa), _tr(transb), m, n, k, float(alpha), A.ctypes.data, lda, B.ctypes.data,
+                                ldb, float(beta), C.ctypes.data, ldc, Chi.ctypes.data, S.ctypes.data, ldo, cptr, ncols)
+    elif dt == np.float32:
+        rc = lib().ref_sgemm_hi(_tr(transa), _tr(transb), m, n, k, float(np.float32(alpha)), A.ctypes.data, lda,
+                                B.ctypes.data, ldb, float(np.float32(beta)), C.ctypes.data, ldc, Chi.ctypes.data,
+                                S.ctypes.data, ldo, cptr, ncols)
+    else:
+        raise TypeError(f"unsupported dtype {dt}")
+    if rc != 0:
+        raise ValueError(f"oracle rejected argument {-rc}")
+    del keep
+    return Chi, S
+
+
+def ref_zgemm_4m(transa, transb, m, n, k, alpha, A, lda, B, ldb, beta, C, ldc) -> None:
+    """Complex GEMM from four real-oracle calls on split planes (4M); C complex128 flat, updated in place.
+
+    A' = alpha*A is formed elementwise in complex arithmetic (each component rounded once), then
+        Cr = A'r*Br - A'i*Bi + (beta*C)r,     Ci = A'r*Bi + A'i*Br + (beta*C)i,
+    each right-hand side evaluated as two real GEMM calls: (alpha=1, beta=0 or 1) followed by
+    (alpha=-1 or +1, beta=1).  With beta == 0 the old C is not read.
+    """
+    alpha, beta = complex(alpha), complex(beta)
+    _flat(A, np.complex128), _flat(B, np.complex128), _flat(C, np.complex128)
+    Av = A.view(np.float64)
+    ar, ai = Av[0::2], Av[1::2]
+    apr = np.ascontiguousarray(alpha.real * ar - alpha.imag * ai)
+    api = np.ascontiguousarray(alpha.real * ai + alpha.imag * ar)
+    Bv = B.view(np.float64)
+    br, bi = np.ascontiguousarray(Bv[0::2]), np.ascontiguousarray(Bv[1::2])
+    Cv = C.view(np.float64)
+    cr0, ci0 = Cv[0::2].copy(), Cv[1::2].copy()
+    if beta == 0:
+        cr, ci, first_beta = np.zeros_like(cr0), np.zeros_like(ci0), 0.0
+    else:
+        cr = np.ascontiguousarray(beta.real * cr0 - beta.imag * ci0)
+        ci = np.ascontiguousarray(beta.real * ci0 + beta.imag * cr0)
+        first_beta = 1.0
+    ref_gemm(transa, transb, m, n, k, 1.0, apr, lda, br, ldb, first_beta, cr, ldc)
+    ref_gemm(transa, transb, m, n, k, -1.0, api, lda, bi, ldb, 1.0, cr, ldc)
+    ref_gemm(transa, transb, m, n, k, 1.0, apr, lda, bi, ldb, first_beta, ci, ldc)
+    ref_gemm(transa, transb, m, n, k, 1.0, api, lda, br, ldb, 1.0, ci, ldc)
+    # write back only the m x n entries the operation owns
+    for j in range(n):
+        s = slice(j * ldc, j * ldc + m)
+        Cv[0::2][s] = cr[s]
+        Cv[1::2][s] = ci[s]

@@ -1,0 +1,237 @@
+/*
+ * CPU oracle for GEMM -- TEST INFRASTRUCTURE, not part of the product.
+ *
+ * Only the tests, the smoke check and the benchmark's CPU-baseline leg may call this file.
+ * It shares no code with the CUDA library and neither includes the other.
+ *
+ * What it computes.  The paper's micro-kernel (Section 2.1, "The micro-kernel") is the sum
+ * of rank-1 updates  C += sum_{p<k} a_p b_p^T.  The method reaches, up to the order of the
+ * floating-point summation, the plain definition of that sum, so the oracle is the
+ * definition written out, with the scaling, transposition and leading dimensions of the
+ * level-3 BLAS statement (which the paper does not restate):
+ *
+ *     acc_ij = sum_{p=0}^{k-1} op(A)_ip * op(B)_pj        (ascending p)
+ *     C_ij   = alpha * acc_ij + beta * C_ij
+ *     op(X) = X or X^T,   column-major  X(r,c) = X[r + c*ldx].
+ *
+ * Rules kept here so a reader can check it by eye:
+ *   - one multiply and one add per term, in the working precision, p ascending, starting
+ *     from zero (compile with -ffp-contract=off: no fused multiply-add, no fast-math);
+ *   - beta == 0: C is not read (C_ij = alpha*acc_ij);  alpha == 0 or k == 0: A and B are not
+ *     read (C_ij = beta*C_ij, or 0 when beta == 0);  alpha == 0 and beta == 1: nothing;
+ *   - only entries (i<m, j<n) of C are touched; padding rows of A, B, C are never read;
+ *   - the only parallelism is OpenMP over columns j, which changes no element's arithmetic;
+ *   - `cols`/`ncols` restrict the work to a list of columns j (NULL = all n columns).
+ *
+ * The *_hi variants accumulate in a wider type (long double for fp64 data, double for fp32
+ * data), return the result in that wider type's nearest working-precision value, and also
+ * return the magnitude sum used by forward error bounds,
+ *     S_ij = |alpha| * sum_p |op(A)_ip| |op(B)_pj| + |beta| |C_ij|.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+static int is_trans(char t) { return t == 'T' || t == 't' || t == 'C' || t == 'c'; }
+static int is_notrans(char t) { return t == 'N' || t == 'n'; }
+
+/* BLAS argument check; returns 0 or the 1-based index of the first illegal argument. */
+static int check_args(char ta, char tb, int64_t m, int64_t n, int64_t k, int64_t lda, int64_t ldb, int64_t ldc) {
+  if (!is_trans(ta) && !is_notrans(ta)) return 1;
+  if (!is_trans(tb) && !is_notrans(tb)) return 2;
+  if (m < 0) return 3;
+  if (n < 0) return 4;
+  if (k < 0) return 5;
+  int64_t rows_a = is_notrans(ta) ? m : k, rows_b = is_notrans(tb) ? k : n;
+  if (lda < (rows_a > 1 ? rows_a : 1)) return 8;
+  if (ldb < (rows_b > 1 ? rows_b : 1)) return 10;
+  if (ldc < (m > 1 ? m : 1)) return 13;
+  return 0;
+}
+
+#define DEFINE_REF_GEMM(NAME, T)                                                                          \
+  int NAME(char transa, char transb, int64_t m, int64_t n, int64_t k, T alpha, const T* A, int64_t lda,    \
+           const T* B, int64_t ldb, T beta, T* C, int64_t ldc, const int64_t* cols, int64_t ncols) {       \
+    int bad = check_args(transa, transb, m, n, k, lda, ldb, ldc);                                          \
+    if (bad) return -bad;                                                                                  \
+    if (m == 0 || n == 0) return 0;                                                                        \
+    if ((alpha == (T)0 || k == 0) && beta == (T)1) return 0;                                               \
+    const int ta = is_trans(transa), tb = is_trans(transb);                                                \
+    const int scale_only = (alpha == (T)0 || k == 0);                                                      \
+    const int64_t nj = cols ? ncols : n;                                                                   \
+    _Pragma("omp parallel for schedule(dynamic, 1)") for (int64_t jj = 0; jj < nj; ++jj) {                 \
+      const int64_t j = cols ? cols[jj] : jj;                                                              \
+      for (int64_t i = 0; i < m; ++i) {                                                                    \
+        T acc = (T)0;                                                                                      \
+        if (!scale_only) {                                                                                 \
+          for (int64_t p = 0; p < k; ++p) {                                                                \
+            const T a = ta ? A[p + i * lda] : A[i + p * lda];                                              \
+            const T b = tb ? B[j + p * ldb] : B[p + j * ldb];                                              \
+            const T prod = a * b;                                                                          \
+            acc = acc + prod;                                                                              \
+          }                                                                                                \
+        }                                                                                                  \
+        T* c = &C[i + j * ldc];                                                                            \
+        if (scale_only) {                                                                                  \
+          *c = (beta == (T)0) ? (T)0 : beta * *c;                                                          \
+        } else if (beta == (T)0) {                                                                         \
+          *c = alpha * acc;                                                                                \
+        } else {                                                                                           \
+          const T t1 = alpha * acc;                                                                        \
+          const T t2 = beta * *c;                                                                          \
+          *c = t1 + t2;                                                                                    \
+        }                                                                                                  \
+      }                                                                                                    \
+    }                                                                                                      \
+    return 0;                                                                                              \
+  }
+
+DEFINE_REF_GEMM(ref_dgemm, double)
+DEFINE_REF_GEMM(ref_sgemm, float)
+
+/* Wide-accumulation variants; Chi receives the rounded wide result, S the magnitude sum. */
+#define DEFINE_REF_GEMM_HI(NAME, T, W, ABSW)                                                              \
+  int NAME(char transa, char transb, int64_t m, int64_t n, int64_t k, T alpha, const T* A, int64_t lda,    \
+           const T* B, int64_t ldb, T beta, const T* C, int64_t ldc, T* Chi, double* S, int64_t ldo,       \
+           const int64_t* cols, int64_t ncols) {                                                           \
+    int bad = check_args(transa, transb, m, n, k, lda, ldb, ldc);                                          \
+    if (bad) return -bad;                                                                                  \
+    if (ldo < (m > 1 ? m : 1)) return -15;                                                                 \
+    if (m == 0 || n == 0) return 0;                                                                        \
+    const int ta = is_trans(transa), tb = is_trans(transb);                                                \
+    const int64_t nj = cols ? ncols : n;                                                                   \
+    _Pragma("omp parallel for schedule(dynamic, 1)") for (int64_t jj = 0; jj < nj; ++jj) {                 \
+      const int64_t j = cols ? cols[jj] : jj;                                                              \
+      for (int64_t i = 0; i < m; ++i) {                                                                    \
+        W acc = 0, mag = 0;                                                                                \
+        if (alpha != (T)0) {                                                                               \
+          for (int64_t p = 0; p < k; ++p) {                                                                \
+            const W a = ta ? A[p + i * lda] : A[i + p * lda];                                              \
+            const W b = tb ? B[j + p * ldb] : B[p + j * ldb];                                              \
+            acc += a * b;                                                                                  \
+            mag += ABSW(a) * ABSW(b);                                                                      \
+          }                                                                                                \
+        }                                                                                                  \
+        W r = (W)alpha * acc, s = ABSW((W)alpha) * mag;                                                    \
+        if (beta != (T)0) {                                                                                \
+          r += (W)beta * (W)C[i + j * ldc];                                                                \
+          s += ABSW((W)beta) * ABSW((W)C[i + j * ldc]);                                                    \
+        }                                                                                                  \
+        Chi[i + j * ldo] = (T)r;                                                                           \
+        S[i + j * ldo] = (double)s;                                                                        \
+      }                                                                                                    \
+    }                                                                                                      \
+    return 0;                                                                                              \
+  }
+
+DEFINE_REF_GEMM_HI(ref_dgemm_hi, double, long double, fabsl)
+DEFINE_REF_GEMM_HI(ref_sgemm_hi, float, double, fabs)
+
+/*
+ * Complex double GEMM by direct complex arithmetic (interleaved re,im; ld in complex
+ * elements).  Each term is the textbook product (ar*br - ai*bi, ar*bi + ai*br) added to the
+ * running sum; the epilogue is the complex alpha*acc + beta*C.  transa/transb: N or T
+ * (plain transpose; the conjugate transpose 'C' is rejected here).
+ * The paper names complex GEMM only as a consumer of the real kernel (Abstract).
+ */
+int ref_zgemm(char transa, char transb, int64_t m, int64_t n, int64_t k, const double* alpha, const double* A,
+              int64_t lda, const double* B, int64_t ldb, const double* beta, double* C, int64_t ldc,
+              const int64_t* cols, int64_t ncols) {
+  if (transa == 'C' || transa == 'c') return -1;
+  if (transb == 'C' || transb == 'c') return -2;
+  int bad = check_args(transa, transb, m, n, k, lda, ldb, ldc);
+  if (bad) return -bad;
+  if (m == 0 || n == 0) return 0;
+  const double alr = alpha[0], ali = alpha[1], ber = beta[0], bei = beta[1];
+  const int alpha0 = (alr == 0.0 && ali == 0.0), beta0 = (ber == 0.0 && bei == 0.0);
+  if ((alpha0 || k == 0) && ber == 1.0 && bei == 0.0) return 0;
+  const int ta = is_trans(transa), tb = is_trans(transb);
+  const int64_t nj = cols ? ncols : n;
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int64_t jj = 0; jj < nj; ++jj) {
+    const int64_t j = cols ? cols[jj] : jj;
+    for (int64_t i = 0; i < m; ++i) {
+      double sr = 0.0, si = 0.0;
+      if (!alpha0) {
+        for (int64_t p = 0; p < k; ++p) {
+          const double* a = ta ? &A[2 * (p + i * lda)] : &A[2 * (i + p * lda)];
+          const double* b = tb ? &B[2 * (j + p * ldb)] : &B[2 * (p + j * ldb)];
+          const double pr = a[0] * b[0] - a[1] * b[1];
+          const double pi = a[0] * b[1] + a[1] * b[0];
+          sr = sr + pr;
+          si = si + pi;
+        }
+      }
+      double* c = &C[2 * (i + j * ldc)];
+      double rr = 0.0, ri = 0.0;
+      if (!alpha0) {
+        rr = alr * sr - ali * si;
+        ri = alr * si + ali * sr;
+      }
+      if (!beta0) {
+        const double cr = c[0], ci = c[1];
+        rr = rr + (ber * cr - bei * ci);
+        ri = ri + (ber * ci + bei * cr);
+      }
+      c[0] = rr;
+      c[1] = ri;
+    }
+  }
+  return 0;
+}
+
+/* Wide (long double) complex GEMM; Chi = rounded result, S = one magnitude sum per element:
+ *   S_ij = (|alr|+|ali|) * sum_p (|Ar|+|Ai|)_ip (|Br|+|Bi|)_pj + (|ber|+|bei|) (|Cr|+|Ci|)_ij,
+ * an upper bound on the magnitude sums of both the real and the imaginary component. */
+int ref_zgemm_hi(char transa, char transb, int64_t m, int64_t n, int64_t k, const double* alpha, const double* A,
+                 int64_t lda, const double* B, int64_t ldb, const double* beta, const double* C, int64_t ldc,
+                 double* Chi, double* S, int64_t ldo, const int64_t* cols, int64_t ncols) {
+  if (transa == 'C' || transa == 'c') return -1;
+  if (transb == 'C' || transb == 'c') return -2;
+  int bad = check_args(transa, transb, m, n, k, lda, ldb, ldc);
+  if (bad) return -bad;
+  if (ldo < (m > 1 ? m : 1)) return -16;
+  if (m == 0 || n == 0) return 0;
+  const long double alr = alpha[0], ali = alpha[1], ber = beta[0], bei = beta[1];
+  const int alpha0 = (alr == 0 && ali == 0), beta0 = (ber == 0 && bei == 0);
+  const int ta = is_trans(transa), tb = is_trans(transb);
+  const int64_t nj = cols ? ncols : n;
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int64_t jj = 0; jj < nj; ++jj) {
+    const int64_t j = cols ? cols[jj] : jj;
+    for (int64_t i = 0; i < m; ++i) {
+      long double sr = 0, si = 0, mag = 0;
+      if (!alpha0) {
+        for (int64_t p = 0; p < k; ++p) {
+          const double* a = ta ? &A[2 * (p + i * lda)] : &A[2 * (i + p * lda)];
+          const double* b = tb ? &B[2 * (j + p * ldb)] : &B[2 * (p + j * ldb)];
+          const long double ar = a[0], ai = a[1], br = b[0], bi = b[1];
+          sr += ar * br - ai * bi;
+          si += ar * bi + ai * br;
+          mag += (fabsl(ar) + fabsl(ai)) * (fabsl(br) + fabsl(bi));
+        }
+      }
+      long double rr = alr * sr - ali * si, ri = alr * si + ali * sr;
+      long double s = (fabsl(alr) + fabsl(ali)) * mag;
+      if (!beta0) {
+        const long double cr = C[2 * (i + j * ldc)], ci = C[2 * (i + j * ldc) + 1];
+        rr += ber * cr - bei * ci;
+        ri += ber * ci + bei * cr;
+        s += (fabsl(ber) + fabsl(bei)) * (fabsl(cr) + fabsl(ci));
+      }
+      Chi[2 * (i + j * ldo)] = (double)rr;
+      Chi[2 * (i + j * ldo) + 1] = (double)ri;
+      S[i + j * ldo] = (double)s;
+    }
+  }
+  return 0;
+}
+
+/* Number of OpenMP threads a parallel region would use (reported beside CPU timings). */
+#ifdef _OPENMP
+#include <omp.h>
+int ref_num_threads(void) { return omp_get_max_threads(); }
+#else
+int ref_num_threads(void) { return 1; }
+#endif
