@@ -1,0 +1,158 @@
+/*
+ * b2gemm -- real GEMM for NVIDIA B200 (sm_100a) computed as a register-blocked sequence of
+ * rank-1 outer-product updates over staged panels of A and B, plus a complex entry built
+ * from four real-kernel calls.
+ *
+ * Source of the operation.  The paper's micro-kernel (Section 2.1, "The micro-kernel") is
+ *     C += A B = sum_{p<kc} a_p b_p^T          (C is mr x nr, A is mr x kc, B is kc x nr)
+ * wrapped in the GotoBLAS/BLIS loop nest (Section 2, Figure 1).  The paper stops at
+ * C += A B; scaling by alpha and beta, transposition, leading dimensions and edge sizes
+ * follow the level-3 BLAS statement of GEMM:
+ *     C := alpha * op(A) * op(B) + beta * C,   op(X) = X or X^T,
+ * with column-major storage, X(r, c) = X[r + c * ldx].
+ *
+ * Conventions shared by every entry point unless its comment says otherwise
+ *   - A, B, C (and any workspace) are DEVICE pointers owned by the caller.  The library
+ *     allocates nothing, keeps no state between calls and never frees anything.
+ *   - Scalars are passed by value from the host.
+ *   - Work is enqueued on `cuda_stream` (a cudaStream_t cast to void*; NULL = the legacy
+ *     default stream) and the call returns without synchronising.
+ *   - trans in {N,n,T,t,C,c}; for real data C means T.
+ *   - m, n, k >= 0;  lda >= max(1, transa==N ? m : k);  ldb >= max(1, transb==N ? k : n);
+ *     ldc >= max(1, m).
+ *   - Return value: 0 on success; -i when the i-th argument is illegal, counted as in the
+ *     reference BLAS: transa 1, transb 2, m 3, n 4, k 5, alpha 6, A 7, lda 8, B 9, ldb 10,
+ *     beta 11, C 12, ldc 13 (nothing is launched); a positive b2_status for run-time failures.
+ *   - Quick returns: m==0 or n==0 does nothing.  alpha==0 or k==0 computes C := beta*C and
+ *     never reads A or B.  beta==0 writes C without reading it (NaN/Inf in the old C do
+ *     not propagate).  alpha==0 and beta==1 does nothing.
+ *   - Rows r >= m of a column of C, and rows of A/B beyond the operand's row count (the
+ *     padding ld - rows), are never written and their contents never influence a result.
+ *   - A and B must not overlap C.
+ *   - Arithmetic: IEEE round-to-nearest, fused multiply-add, denormals kept; fp32 entries
+ *     use FP32 FMA only (no TF32).  The order of the k-summation is unspecified.
+ */
+#ifndef B2GEMM_H_
+#define B2GEMM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  B2_OK = 0,
+  B2_ERR_TIMEOUT = 1001,   /* a bounded device-side wait gave up */
+  B2_ERR_LAUNCH = 1002,    /* the CUDA runtime refused a launch or a copy */
+  B2_ERR_WORKSPACE = 1003, /* workspace pointer null, misaligned or too small */
+  B2_ERR_VARIANT = 1004    /* unknown or inapplicable kernel variant */
+} b2_status;
+
+/* Kernel variants (micro-kernel x tile).  B2_VARIANT_AUTO lets the analytic selector choose. */
+#define B2_VARIANT_AUTO (-1)
+
+/*
+ * Double-precision GEMM, C := alpha*op(A)*op(B) + beta*C  (micro-kernel sum of Section 2.1;
+ * BLAS semantics as stated at the top of this file).  All pointers are device pointers.
+ */
+int b2_dgemm(char transa, char transb, int64_t m, int64_t n, int64_t k, double alpha, const double* A,
+             int64_t lda, const double* B, int64_t ldb, double beta, double* C, int64_t ldc,
+             void* cuda_stream);
+
+/* Single-precision GEMM, same definition; FP32 FMA arithmetic only. */
+int b2_sgemm(char transa, char transb, int64_t m, int64_t n, int64_t k, float alpha, const float* A,
+             int64_t lda, const float* B, int64_t ldb, float beta, float* C, int64_t ldc,
+             void* cuda_stream);
+
+/*
+ * The same two operations with an explicit kernel variant, 0 <= variant < b2_variant_count(dtype),
+ * or B2_VARIANT_AUTO.  Used by tests and benchmarks to exercise every micro-kernel; a variant
+ * that cannot serve the given shape/alignment returns B2_ERR_VARIANT and launches nothing.
+ */
+int b2_dgemm_variant(int variant, char transa, char transb, int64_t m, int64_t n, int64_t k, double alpha,
+                     const double* A, int64_t lda, const double* B, int64_t ldb, double beta, double* C,
+                     int64_t ldc, void* cuda_stream);
+int b2_sgemm_variant(int variant, char transa, char transb, int64_t m, int64_t n, int64_t k, float alpha,
+                     const float* A, int64_t lda, const float* B, int64_t ldb, float beta, float* C,
+                     int64_t ldc, void* cuda_stream);
+
+/* dtype codes for the query calls */
+#define B2_F64 0
+#define B2_F32 1
+
+/* Number of kernel variants for a dtype, and a static, NUL-terminated description of one
+ * ("dmma_128x128x16_s4" ...); NULL when out of range. */
+int b2_variant_count(int dtype);
+const char* b2_variant_name(int dtype, int variant);
+
+/*
+ * Writes a NUL-terminated JSON object describing what the selector would launch for this
+ * problem (variant, CTA tile, kc, stages, micro-kernel, grid, shared memory) into json_out
+ * (HOST memory, capacity cap bytes).  Returns 0, a negative argument index as above (dtype is
+ * argument 1 here, the rest shift by one), or B2_ERR_WORKSPACE when cap is too small.
+ * Nothing is launched.  The tile derivation follows the paper's register-limit formula
+ * (Section 5, "Limits imposed by registers") and pipeline-throughput estimate (Section 4).
+ */
+int b2_gemm_query_config(int dtype, char transa, char transb, int64_t m, int64_t n, int64_t k, int64_t lda,
+                         int64_t ldb, int64_t ldc, char* json_out, size_t cap);
+
+/*
+ * Complex double GEMM (interleaved re,im; column-major; leading dimensions in complex
+ * elements) built from four real-kernel launches ("4M"): the paper names complex GEMM only
+ * as a consumer of the real kernel (Abstract).  With A' = alpha*A rounded once per component,
+ *     Cr = A'r*Br - A'i*Bi + (beta*C)r,   Ci = A'r*Bi + A'i*Br + (beta*C)i.
+ * alpha and beta point to HOST {re, im} pairs.  transa/transb accept N and T (C, the
+ * conjugate transpose, is rejected with -1/-2).  workspace is DEVICE memory of at least
+ * b2_zgemm4m_workspace_bytes(...) bytes, 256-byte aligned, owned by the caller; its contents
+ * are overwritten.  Argument numbering as above with workspace = 14.
+ */
+size_t b2_zgemm4m_workspace_bytes(char transa, char transb, int64_t m, int64_t n, int64_t k);
+int b2_zgemm4m(char transa, char transb, int64_t m, int64_t n, int64_t k, const double alpha[2], const void* A,
+               int64_t lda, const void* B, int64_t ldb, const double beta[2], void* C, int64_t ldc,
+               void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Host-buffer forms: A, B, C are HOST pointers (pinned memory makes the copies asynchronous),
+ * dev_workspace is DEVICE memory of at least b2_gemm_host_workspace_bytes(...) bytes owned by
+ * the caller.  The call copies the referenced parts of A and B (and C when beta != 0) to the
+ * device, runs the same kernel as b2_dgemm / b2_sgemm, copies the m x n result back into C and
+ * synchronises the stream before returning.  Argument numbering as b2_dgemm, workspace = 14.
+ */
+size_t b2_gemm_host_workspace_bytes(int dtype, char transa, char transb, int64_t m, int64_t n, int64_t k);
+int b2_dgemm_host(char transa, char transb, int64_t m, int64_t n, int64_t k, double alpha, const double* A,
+                  int64_t lda, const double* B, int64_t ldb, double beta, double* C, int64_t ldc,
+                  void* dev_workspace, size_t workspace_bytes, void* cuda_stream);
+int b2_sgemm_host(char transa, char transb, int64_t m, int64_t n, int64_t k, float alpha, const float* A,
+                  int64_t lda, const float* B, int64_t ldb, float beta, float* C, int64_t ldc,
+                  void* dev_workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Pipeline-throughput probe (Section 4, "Estimating throughput": the estimate needs each
+ * pipeline's rate).  Launches `ctas` CTAs of `threads_per_cta` threads that each issue
+ * `iters` rounds of independent register-resident multiply-adds of the given kind and
+ * returns.  scratch is DEVICE memory of at least 64 + 8*ctas bytes; after the stream has
+ * drained, the int64 at byte offset 64 + 8*b holds the SM clock cycles CTA b spent in the
+ * loop.  *fma_per_thread_iter (HOST) receives the multiply-adds one thread performs per round,
+ * so rate = threads * iters * (*fma_per_thread_iter) / cycles.  Returns 0, -i for a bad
+ * i-th argument, or B2_ERR_LAUNCH.
+ */
+#define B2_PROBE_DFMA 0
+#define B2_PROBE_FFMA 1
+#define B2_PROBE_DMMA_M8N8K4 2
+#define B2_PROBE_DMMA_M16N8K4 3
+#define B2_PROBE_DMMA_M16N8K8 4
+#define B2_PROBE_DMMA_M16N8K16 5
+int b2_pipe_probe(int kind, int threads_per_cta, int ctas, int64_t iters, void* scratch, size_t scratch_bytes,
+                  double* fma_per_thread_iter, void* cuda_stream);
+
+/* Static, NUL-terminated text for a return value of any call above. */
+const char* b2_strerror(int status);
+/* Static, NUL-terminated library version. */
+const char* b2_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* B2GEMM_H_ */

@@ -1,0 +1,188 @@
+"""ctypes binding of ``libb2gemm.so``: argument marshalling only.
+
+Each Python function has the name and argument order of the C entry point it wraps (see
+``include/b2gemm.h``); tensors are passed as raw device (or host) pointers plus sizes, the
+stream as ``torch.cuda.current_stream().cuda_stream``.  No arithmetic of the GEMM happens
+here.  Loading fails loudly when the library has not been built: there is no fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+from ctypes import c_char, c_char_p, c_double, c_float, c_int, c_int64, c_size_t, c_void_p
+from pathlib import Path
+
+import torch
+
+LIB_PATH = Path(__file__).resolve().parent / "libb2gemm.so"
+_lib = None
+
+_GEMM_TAIL_D = [c_char, c_char, c_int64, c_int64, c_int64, c_double, c_void_p, c_int64, c_void_p, c_int64, c_double,
+                c_void_p, c_int64]
+_GEMM_TAIL_S = [c_char, c_char, c_int64, c_int64, c_int64, c_float, c_void_p, c_int64, c_void_p, c_int64, c_float,
+                c_void_p, c_int64]
+
+_SIGNATURES = {
+    "b2_dgemm": (c_int, _GEMM_TAIL_D + [c_void_p]),
+    "b2_sgemm": (c_int, _GEMM_TAIL_S + [c_void_p]),
+    "b2_dgemm_variant": (c_int, [c_int] + _GEMM_TAIL_D + [c_void_p]),
+    "b2_sgemm_variant": (c_int, [c_int] + _GEMM_TAIL_S + [c_void_p]),
+    "b2_variant_count": (c_int, [c_int]),
+    "b2_variant_name": (c_char_p, [c_int, c_int]),
+    "b2_gemm_query_config": (c_int, [c_int, c_char, c_char, c_int64, c_int64, c_int64, c_int64, c_int64, c_int64,
+                                     c_char_p, c_size_t]),
+    "b2_zgemm4m_workspace_bytes": (c_size_t, [c_char, c_char, c_int64, c_int64, c_int64]),
+    "b2_zgemm4m": (c_int, [c_char, c_char, c_int64, c_int64, c_int64, ctypes.POINTER(c_double), c_void_p, c_int64,
+                           c_void_p, c_int64, ctypes.POINTER(c_double), c_void_p, c_int64, c_void_p, c_size_t,
+                           c_void_p]),
+    "b2_gemm_host_workspace_bytes": (c_size_t, [c_int, c_char, c_char, c_int64, c_int64, c_int64]),
+    "b2_dgemm_host": (c_int, _GEMM_TAIL_D + [c_void_p, c_size_t, c_void_p]),
+    "b2_sgemm_host": (c_int, _GEMM_TAIL_S + [c_void_p, c_size_t, c_void_p]),
+    "b2_pipe_probe": (c_int, [c_int, c_int, c_int, c_int64, c_void_p, c_size_t, ctypes.POINTER(c_double), c_void_p]),
+    "b2_strerror": (c_char_p, [c_int]),
+    "b2_version": (c_char_p, []),
+}
+
+EXPORTED_SYMBOLS = tuple(_SIGNATURES)
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded C library (loaded once).  Raises when it has not been built."""
+    global _lib
+    if _lib is None:
+        if not LIB_PATH.exists():
+            raise RuntimeError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_1611_08035_b200.build` "
+                "(there is no CPU or library fallback)")
+        handle = ctypes.CDLL(str(LIB_PATH))
+        for name, (res, args) in _SIGNATURES.items():
+            fn = getattr(handle, name)
+            fn.restype = res
+            fn.argtypes = args
+        _lib = handle
+    return _lib
+
+
+def strerror(status: int) -> str:
+    return lib().b2_strerror(int(status)).decode()
+
+
+def version() -> str:
+    return lib().b2_version().decode()
+
+
+class B2Error(RuntimeError):
+    def __init__(self, fn: str, status: int):
+        super().__init__(f"{fn} returned {status}: {strerror(status)}")
+        self.status = status
+
+
+def _tr(c: str) -> bytes:
+    return c.encode("ascii")[:1]
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _check(fn: str, rc: int) -> None:
+    if rc != 0:
+        raise B2Error(fn, rc)
+
+
+def _ptr(t) -> int:
+    return 0 if t is None else t.data_ptr()
+
+
+def b2_dgemm(transa, transb, m, n, k, alpha, A, lda, B, ldb, beta, C, ldc, variant=None, check=True) -> int:
+    """C := alpha*op(A)*op(B) + beta*C in fp64 on device tensors (column-major storage)."""
+    for t in (A, B, C):
+        if t is not None and (t.dtype != torch.float64 or not t.is_cuda):
+            raise TypeError("b2_dgemm takes float64 CUDA tensors")
+    if variant is None:
+        rc = lib().b2_dgemm(_tr(transa), _tr(transb), m, n, k, alpha, _ptr(A), lda, _ptr(B), ldb, beta, _ptr(C), ldc,
+                            _stream())
+    else:
+        rc = lib().b2_dgemm_variant(variant, _tr(transa), _tr(transb), m, n, k, alpha, _ptr(A), lda, _ptr(B), ldb,
+                                    beta, _ptr(C), ldc, _stream())
+    if check:
+        _check("b2_dgemm", rc)
+    return rc
+
+
+def b2_sgemm(transa, transb, m, n, k, alpha, A, lda, B, ldb, beta, C, ldc, variant=None, check=True) -> int:
+    """C := alpha*op(A)*op(B) + beta*C in fp32 (FP32 FMA only) on device tensors."""
+    for t in (A, B, C):
+        if t is not None and (t.dtype != torch.float32 or not t.is_cuda):
+            raise TypeError("b2_sgemm takes float32 CUDA tensors")
+    if variant is None:
+        rc = lib().b2_sgemm(_tr(transa), _tr(transb), m, n, k, alpha, _ptr(A), lda, _ptr(B), ldb, beta, _ptr(C), ldc,
+                            _stream())
+    else:
+        rc = lib().b2_sgemm_variant(variant, _tr(transa), _tr(transb), m, n, k, alpha, _ptr(A), lda, _ptr(B), ldb,
+                                    beta, _ptr(C), ldc, _stream())
+    if check:
+        _check("b2_sgemm", rc)
+    return rc
+
+
+def b2_variant_count(dtype: int) -> int:
+    return lib().b2_variant_count(dtype)
+
+
+def b2_variant_name(dtype: int, variant: int):
+    s = lib().b2_variant_name(dtype, variant)
+    return None if s is None else s.decode()
+
+
+def b2_gemm_query_config(dtype, transa, transb, m, n, k, lda, ldb, ldc) -> str:
+    buf = ctypes.create_string_buffer(1024)
+    rc = lib().b2_gemm_query_config(dtype, _tr(transa), _tr(transb), m, n, k, lda, ldb, ldc, buf, len(buf))
+    _check("b2_gemm_query_config", rc)
+    return buf.value.decode()
+
+
+def b2_zgemm4m_workspace_bytes(transa, transb, m, n, k) -> int:
+    return lib().b2_zgemm4m_workspace_bytes(_tr(transa), _tr(transb), m, n, k)
+
+
+def b2_zgemm4m(transa, transb, m, n, k, alpha, A, lda, B, ldb, beta, C, ldc, workspace, check=True) -> int:
+    """Complex128 GEMM from four real-kernel launches; A, B, C complex128 CUDA tensors, workspace uint8."""
+    for t in (A, B, C):
+        if t is not None and (t.dtype != torch.complex128 or not t.is_cuda):
+            raise TypeError("b2_zgemm4m takes complex128 CUDA tensors")
+    al = (c_double * 2)(complex(alpha).real, complex(alpha).imag)
+    be = (c_double * 2)(complex(beta).real, complex(beta).imag)
+    wbytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    rc = lib().b2_zgemm4m(_tr(transa), _tr(transb), m, n, k, al, _ptr(A), lda, _ptr(B), ldb, be, _ptr(C), ldc,
+                          _ptr(workspace), wbytes, _stream())
+    if check:
+        _check("b2_zgemm4m", rc)
+    return rc
+
+
+def b2_gemm_host_workspace_bytes(dtype, transa, transb, m, n, k) -> int:
+    return lib().b2_gemm_host_workspace_bytes(dtype, _tr(transa), _tr(transb), m, n, k)
+
+
+def _host_call(fn_name, want, transa, transb, m, n, k, alpha, A, lda, B, ldb, beta, C, ldc, workspace, check):
+    for t in (A, B, C):
+        if t is not None and (t.dtype != want or t.is_cuda):
+            raise TypeError(f"{fn_name} takes {want} HOST tensors")
+    wbytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    rc = getattr(lib(), fn_name)(_tr(transa), _tr(transb), m, n, k, alpha, _ptr(A), lda, _ptr(B), ldb, beta, _ptr(C),
+                                 ldc, _ptr(workspace), wbytes, _stream())
+    if check:
+        _check(fn_name, rc)
+    return rc
+
+
+def b2_dgemm_host(transa, transb, m, n, k, alpha, A, lda, B, ldb, beta, C, ldc, workspace, check=True) -> int:
+    """b2_dgemm on HOST tensors (pinned for speed); copies in, computes on the GPU, copies C back."""
+    return _host_call("b2_dgemm_host", torch.float64, transa, transb, m, n, k, alpha, A, lda, B, ldb, beta, C, ldc,
+                      workspace, check)
+
+
+def b2_sgemm_host(transa, transb, m, n, k, alpha, A, lda, B, ldb, beta, C, ldc, workspace, check=True) -> int:
+    """b2_sgemm on HOST tensors (pinned for speed); copies in, computes on the GPU, copies C back."""
+    return _host_call("b2_sgemm_host", torch.float32, transa, transb, m, n, k, alpha, A, lda, B, ldb, beta, C, ldc,
+                      workspace, check)

@@ -1,0 +1,244 @@
+// C-ABI entry points of the real GEMM: argument checking, quick returns, variant selection.
+#include <cuda_runtime.h>
+#include <stdio.h>
+#include <string.h>
+
+#include "b2gemm.h"
+#include "entry.h"
+#include "gemm_launch.cuh"
+#include "select.h"
+
+namespace b2 {
+
+int launch_f64_v0(const GemmArgs<double>&, bool, bool, bool, cudaStream_t);
+int launch_f64_v1(const GemmArgs<double>&, bool, bool, bool, cudaStream_t);
+int launch_f64_v2(const GemmArgs<double>&, bool, bool, bool, cudaStream_t);
+int launch_f64_v3(const GemmArgs<double>&, bool, bool, bool, cudaStream_t);
+int launch_f32_v0(const GemmArgs<float>&, bool, bool, bool, cudaStream_t);
+int launch_f32_v1(const GemmArgs<float>&, bool, bool, bool, cudaStream_t);
+int launch_f32_v2(const GemmArgs<float>&, bool, bool, bool, cudaStream_t);
+
+namespace {
+
+// name, micro-kernel, BM, BN, BK, stages, threads, resident CTAs per SM
+const VariantInfo kF64Info[] = {
+    {"dmma_128x128x16_s4", "dmma", 128, 128, 16, 4, 256, 1},
+    {"dmma_128x64x16_s3", "dmma", 128, 64, 16, 3, 128, 2},
+    {"dmma_64x64x16_s3", "dmma", 64, 64, 16, 3, 128, 4},
+    {"dfma_128x64x16_s3", "dfma", 128, 64, 16, 3, 128, 2},
+};
+const LaunchFn<double> kF64Launch[] = {launch_f64_v0, launch_f64_v1, launch_f64_v2, launch_f64_v3};
+const VariantInfo kF32Info[] = {
+    {"ffma_128x128x16_s4", "ffma", 128, 128, 16, 4, 256, 2},
+    {"ffma_128x64x16_s4", "ffma", 128, 64, 16, 4, 128, 4},
+    {"ffma_64x64x16_s4", "ffma", 64, 64, 16, 4, 64, 8},
+};
+const LaunchFn<float> kF32Launch[] = {launch_f32_v0, launch_f32_v1, launch_f32_v2};
+
+}  // namespace
+
+int f64_variant_count() { return (int)(sizeof(kF64Info) / sizeof(kF64Info[0])); }
+const VariantInfo& f64_variant_info(int v) { return kF64Info[v]; }
+LaunchFn<double> f64_variant_launch(int v) { return kF64Launch[v]; }
+int f32_variant_count() { return (int)(sizeof(kF32Info) / sizeof(kF32Info[0])); }
+const VariantInfo& f32_variant_info(int v) { return kF32Info[v]; }
+LaunchFn<float> f32_variant_launch(int v) { return kF32Launch[v]; }
+
+static bool is_n(char c) { return c == 'N' || c == 'n'; }
+static bool is_t(char c) { return c == 'T' || c == 't' || c == 'C' || c == 'c'; }
+
+// BLAS argument check; 0 or the negative index of the first illegal argument.
+int check_gemm_args(char transa, char transb, int64_t m, int64_t n, int64_t k, const void* A, int64_t lda,
+                    const void* B, int64_t ldb, const void* C, int64_t ldc, bool reads_ab) {
+  if (!is_n(transa) && !is_t(transa)) return -1;
+  if (!is_n(transb) && !is_t(transb)) return -2;
+  if (m < 0) return -3;
+  if (n < 0) return -4;
+  if (k < 0) return -5;
+  const int64_t rows_a = is_n(transa) ? m : k, rows_b = is_n(transb) ? k : n;
+  const bool nonempty = m > 0 && n > 0;
+  if (nonempty && reads_ab && !A) return -7;
+  if (lda < (rows_a > 1 ? rows_a : 1)) return -8;
+  if (nonempty && reads_ab && !B) return -9;
+  if (ldb < (rows_b > 1 ? rows_b : 1)) return -10;
+  if (nonempty && !C) return -12;
+  if (ldc < (m > 1 ? m : 1)) return -13;
+  return 0;
+}
+
+static int sm_count_cached() {
+  static int cached[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+  if (cached[dev] == 0) {
+    int sms = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) sms = 148;
+    cached[dev] = sms;
+  }
+  return cached[dev];
+}
+
+template <typename T>
+static int variant_count_t();
+template <>
+int variant_count_t<double>() { return f64_variant_count(); }
+template <>
+int variant_count_t<float>() { return f32_variant_count(); }
+template <typename T>
+static const VariantInfo& variant_info_t(int v);
+template <>
+const VariantInfo& variant_info_t<double>(int v) { return f64_variant_info(v); }
+template <>
+const VariantInfo& variant_info_t<float>(int v) { return f32_variant_info(v); }
+template <typename T>
+static LaunchFn<T> variant_launch_t(int v);
+template <>
+LaunchFn<double> variant_launch_t<double>(int v) { return f64_variant_launch(v); }
+template <>
+LaunchFn<float> variant_launch_t<float>(int v) { return f32_variant_launch(v); }
+
+template <typename T>
+static bool operands_aligned(const T* A, int64_t lda, const T* B, int64_t ldb) {
+  constexpr int VEC = 16 / (int)sizeof(T);
+  return ((reinterpret_cast<uintptr_t>(A) & 15) == 0) && ((reinterpret_cast<uintptr_t>(B) & 15) == 0) &&
+         (lda % VEC == 0) && (ldb % VEC == 0);
+}
+
+template <typename T>
+int choose_variant(int64_t m, int64_t n, int64_t k) {
+  const int count = variant_count_t<T>();
+  TileChoice cand[16];
+  for (int v = 0; v < count && v < 16; ++v) {
+    const VariantInfo& vi = variant_info_t<T>(v);
+    cand[v] = TileChoice{vi.bm, vi.bn, vi.bk, vi.threads, vi.ctas_per_sm, strcmp(vi.micro, "dfma") == 0};
+  }
+  return select_tile(cand, count < 16 ? count : 16, m, n, k, sm_count_cached(), (int)sizeof(T));
+}
+
+template <typename T>
+int gemm_entry(int variant, char transa, char transb, int64_t m, int64_t n, int64_t k, T alpha, const T* A,
+               int64_t lda, const T* B, int64_t ldb, T beta, T* C, int64_t ldc, void* cuda_stream) {
+  const bool scale_only = (alpha == T(0) || k == 0);
+  const int bad = check_gemm_args(transa, transb, m, n, k, A, lda, B, ldb, C, ldc, !scale_only);
+  if (bad) return bad;
+  if (variant != B2_VARIANT_AUTO && (variant < 0 || variant >= variant_count_t<T>())) return B2_ERR_VARIANT;
+  if (m == 0 || n == 0) return B2_OK;
+  cudaStream_t stream = (cudaStream_t)cuda_stream;
+  if (scale_only) {
+    if (beta == T(1)) return B2_OK;
+    const int64_t total = m * n;
+    const int threads = 256;
+    int64_t blocks = (total + threads - 1) / threads;
+    const int64_t cap = (int64_t)sm_count_cached() * 16;
+    if (blocks > cap) blocks = cap;
+    scale_kernel<T><<<(unsigned)blocks, threads, 0, stream>>>(m, n, beta, C, ldc);
+    return cudaGetLastError() == cudaSuccess ? B2_OK : B2_ERR_LAUNCH;
+  }
+  if (variant == B2_VARIANT_AUTO) variant = choose_variant<T>(m, n, k);
+  GemmArgs<T> args;
+  args.m = m, args.n = n, args.k = k;
+  args.alpha = alpha, args.beta = beta;
+  args.A = A, args.lda = lda, args.B = B, args.ldb = ldb, args.C = C, args.ldc = ldc;
+  args.tiles_m = args.tiles_n = 0;
+  args.group_m = 8;
+  return variant_launch_t<T>(variant)(args, is_t(transa), is_t(transb), operands_aligned(A, lda, B, ldb), stream);
+}
+
+// Explicit instantiations used by the other translation units (complex and host-buffer entries).
+template int gemm_entry<double>(int, char, char, int64_t, int64_t, int64_t, double, const double*, int64_t,
+                                const double*, int64_t, double, double*, int64_t, void*);
+template int gemm_entry<float>(int, char, char, int64_t, int64_t, int64_t, float, const float*, int64_t, const float*,
+                               int64_t, float, float*, int64_t, void*);
+
+}  // namespace b2
+
+extern "C" int b2_dgemm(char transa, char transb, int64_t m, int64_t n, int64_t k, double alpha, const double* A,
+                        int64_t lda, const double* B, int64_t ldb, double beta, double* C, int64_t ldc,
+                        void* cuda_stream) {
+  return b2::gemm_entry<double>(B2_VARIANT_AUTO, transa, transb, m, n, k, alpha, A, lda, B, ldb, beta, C, ldc,
+                                cuda_stream);
+}
+
+extern "C" int b2_sgemm(char transa, char transb, int64_t m, int64_t n, int64_t k, float alpha, const float* A,
+                        int64_t lda, const float* B, int64_t ldb, float beta, float* C, int64_t ldc,
+                        void* cuda_stream) {
+  return b2::gemm_entry<float>(B2_VARIANT_AUTO, transa, transb, m, n, k, alpha, A, lda, B, ldb, beta, C, ldc,
+                               cuda_stream);
+}
+
+extern "C" int b2_dgemm_variant(int variant, char transa, char transb, int64_t m, int64_t n, int64_t k, double alpha,
+                                const double* A, int64_t lda, const double* B, int64_t ldb, double beta, double* C,
+                                int64_t ldc, void* cuda_stream) {
+  return b2::gemm_entry<double>(variant, transa, transb, m, n, k, alpha, A, lda, B, ldb, beta, C, ldc, cuda_stream);
+}
+
+extern "C" int b2_sgemm_variant(int variant, char transa, char transb, int64_t m, int64_t n, int64_t k, float alpha,
+                                const float* A, int64_t lda, const float* B, int64_t ldb, float beta, float* C,
+                                int64_t ldc, void* cuda_stream) {
+  return b2::gemm_entry<float>(variant, transa, transb, m, n, k, alpha, A, lda, B, ldb, beta, C, ldc, cuda_stream);
+}
+
+extern "C" int b2_variant_count(int dtype) {
+  if (dtype == B2_F64) return b2::f64_variant_count();
+  if (dtype == B2_F32) return b2::f32_variant_count();
+  return 0;
+}
+
+extern "C" const char* b2_variant_name(int dtype, int variant) {
+  if (variant < 0 || variant >= b2_variant_count(dtype)) return nullptr;
+  return dtype == B2_F64 ? b2::f64_variant_info(variant).name : b2::f32_variant_info(variant).name;
+}
+
+extern "C" int b2_gemm_query_config(int dtype, char transa, char transb, int64_t m, int64_t n, int64_t k, int64_t lda,
+                                    int64_t ldb, int64_t ldc, char* json_out, size_t cap) {
+  if (dtype != B2_F64 && dtype != B2_F32) return -1;
+  // dummy non-null pointers: only sizes and leading dimensions are checked here
+  const void* dummy = reinterpret_cast<const void*>(16);
+  const int bad = b2::check_gemm_args(transa, transb, m, n, k, dummy, lda, dummy, ldb, dummy, ldc, true);
+  if (bad) return bad - 1;
+  if (!json_out) return -11;
+  const int v = dtype == B2_F64 ? b2::choose_variant<double>(m, n, k) : b2::choose_variant<float>(m, n, k);
+  const b2::VariantInfo& vi = dtype == B2_F64 ? b2::f64_variant_info(v) : b2::f32_variant_info(v);
+  const long long tiles_m = (m + vi.bm - 1) / vi.bm, tiles_n = (n + vi.bn - 1) / vi.bn;
+  const int elem = dtype == B2_F64 ? 8 : 4;
+  const bool ld_aligned = (lda % (16 / elem) == 0) && (ldb % (16 / elem) == 0);
+  char buf[768];
+  const int len = snprintf(
+      buf, sizeof(buf),
+      "{\"dtype\": \"%s\", \"variant\": %d, \"name\": \"%s\", \"micro_kernel\": \"%s\", \"BM\": %d, \"BN\": %d, "
+      "\"kc\": %d, \"stages\": %d, \"threads\": %d, \"ctas_per_sm\": %d, \"grid\": %lld, \"tiles_m\": %lld, "
+      "\"tiles_n\": %lld, \"k_slabs\": %lld, \"vector_staging_if_pointers_aligned\": %s, \"sm_count\": %d}",
+      dtype == B2_F64 ? "f64" : "f32", v, vi.name, vi.micro, vi.bm, vi.bn, vi.bk, vi.stages, vi.threads,
+      vi.ctas_per_sm, tiles_m * tiles_n, tiles_m, tiles_n, (long long)((k + vi.bk - 1) / vi.bk),
+      ld_aligned ? "true" : "false", b2::sm_count_cached());
+  if (len < 0 || (size_t)len + 1 > cap) return B2_ERR_WORKSPACE;
+  memcpy(json_out, buf, (size_t)len + 1);
+  return B2_OK;
+}
+
+extern "C" const char* b2_version(void) { return "b2gemm 0.1 (sm_100a)"; }
+
+extern "C" const char* b2_strerror(int status) {
+  switch (status) {
+    case B2_OK: return "success";
+    case B2_ERR_TIMEOUT: return "a bounded device-side wait gave up";
+    case B2_ERR_LAUNCH: return "CUDA launch or copy failed";
+    case B2_ERR_WORKSPACE: return "workspace or output buffer null, misaligned or too small";
+    case B2_ERR_VARIANT: return "unknown or inapplicable kernel variant";
+    case -1: return "argument 1 is illegal";
+    case -2: return "argument 2 is illegal";
+    case -3: return "argument 3 is illegal";
+    case -4: return "argument 4 is illegal";
+    case -5: return "argument 5 is illegal";
+    case -6: return "argument 6 is illegal";
+    case -7: return "argument 7 is illegal";
+    case -8: return "argument 8 is illegal";
+    case -9: return "argument 9 is illegal";
+    case -10: return "argument 10 is illegal";
+    case -11: return "argument 11 is illegal";
+    case -12: return "argument 12 is illegal";
+    case -13: return "argument 13 is illegal";
+    case -14: return "argument 14 is illegal";
+    default: return status < 0 ? "illegal argument" : "unknown status";
+  }
+}

@@ -1,0 +1,65 @@
+// Shared device helpers: kernel arguments, cp.async wrappers, tile rasterisation.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace b2 {
+
+// Arguments of one real GEMM launch, C := alpha*op(A)*op(B) + beta*C (column-major).
+// op() is folded into the kernel's template parameters; m, n, k are the BLAS sizes.
+template <typename T>
+struct GemmArgs {
+  int64_t m, n, k;
+  T alpha, beta;
+  const T* A;
+  int64_t lda;
+  const T* B;
+  int64_t ldb;
+  T* C;
+  int64_t ldc;
+  int tiles_m, tiles_n;  // CTA-tile counts along m and n
+  int group_m;           // rasterisation: tile rows per group
+};
+
+// ---- cp.async (global -> shared, asynchronous, zero-filling past src_bytes) -------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+
+template <int BYTES>
+__device__ __forceinline__ void cp_async_zfill(void* smem_dst, const void* gmem_src, int src_bytes) {
+  static_assert(BYTES == 4 || BYTES == 8 || BYTES == 16, "cp.async copies 4, 8 or 16 bytes");
+  if constexpr (BYTES == 16) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(smem_u32(smem_dst)), "l"(gmem_src),
+                 "r"(src_bytes)
+                 : "memory");
+  } else {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], %2, %3;\n" ::"r"(smem_u32(smem_dst)), "l"(gmem_src),
+                 "n"(BYTES), "r"(src_bytes)
+                 : "memory");
+  }
+}
+
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
+
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+  asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory");
+}
+
+// ---- tile rasterisation ---------------------------------------------------------------
+// Linear CTA index -> (tile row, tile column).  Tiles are visited in groups of `group_m` tile
+// rows, column by column inside a group, so that the CTAs resident at one time cover a
+// compact block of C and share their A row-panels and B column-panels in L2 (the role the
+// nc/mc loops play in the paper's Figure 1 loop nest).
+__device__ __forceinline__ void tile_coords(int linear, int tiles_m, int tiles_n, int group_m, int& tm, int& tn) {
+  const int per_group = group_m * tiles_n;
+  const int group = linear / per_group;
+  const int first_m = group * group_m;
+  const int rows = min(group_m, tiles_m - first_m);
+  const int in_group = linear - group * per_group;
+  tn = in_group / rows;
+  tm = first_m + (in_group - tn * rows);
+}
+
+}  // namespace b2

@@ -1,0 +1,19 @@
+// Internal declarations shared by the translation units that implement C-ABI entry points.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace b2 {
+
+// Real GEMM behind b2_dgemm / b2_sgemm (argument check, quick returns, variant choice, launch).
+template <typename T>
+int gemm_entry(int variant, char transa, char transb, int64_t m, int64_t n, int64_t k, T alpha, const T* A,
+               int64_t lda, const T* B, int64_t ldb, T beta, T* C, int64_t ldc, void* cuda_stream);
+
+// BLAS argument check; 0 or the negative 1-based index of the first illegal argument.
+int check_gemm_args(char transa, char transb, int64_t m, int64_t n, int64_t k, const void* A, int64_t lda,
+                    const void* B, int64_t ldb, const void* C, int64_t ldc, bool reads_ab);
+
+inline size_t round_up(size_t x, size_t to) { return (x + to - 1) / to * to; }
+
+}  // namespace b2

@@ -1,0 +1,418 @@
+// The GEMM kernel: blocked loop nest, shared-memory staging ("packing"), micro-kernel,
+// fringe handling and the fused alpha/beta epilogue.
+//
+// Structure, following the paper:
+//   - Section 2 / Figure 1 (GotoBLAS loop nest as refactored in BLIS): the loops over column
+//     panels and row panels of C become the grid of CTA tiles (BM x BN); the kc loop becomes
+//     the CTA's loop over BK-deep slabs; packing into per-cache-level buffers becomes a
+//     multi-stage cp.async ring in shared memory.
+//   - Section 2.1: inside a tile, C(mr x nr) += sum_p a_p b_p^T on register-resident
+//     accumulators.  Section 5 (kernel skeleton): zero the accumulators, run the unrolled
+//     k-loop of outer products, then add the accumulators into C.
+//   - Section 4 ("Dealing with dependencies across pipelines"): the accumulator tile is
+//     sized so that every multiply-add of one outer product is independent.
+// What the paper leaves out (alpha, beta, transposes, leading dimensions, edge tiles) follows
+// the BLAS definition of GEMM.
+#pragma once
+#include <type_traits>
+
+#include "common.cuh"
+
+namespace b2 {
+
+// Shared-memory layout of a staged operand tile (BO "outer" rows/columns of C by BK of k).
+//   OC: [k][o], o contiguous (pitch in elements) -- the paper's packed micro-panel layout
+//       (A column-major mr x kc, B row-major kc x nr).
+//   KC: [o][k], k contiguous -- the source layout of a transposed A or a non-transposed B,
+//       which the tensor-core fragment loads can read directly.
+enum Layout { OC = 0, KC = 1 };
+
+// ---------------------------------------------------------------------------------------
+// Staging of one BO x BK operand tile from global memory into shared memory with cp.async.
+// X0 points at element (o0, k0) of the operand; o_valid / k_valid are the numbers of valid
+// rows and k-entries from there (anything beyond is zero-filled and never read from global).
+// VEC is the number of elements per cp.async when source and destination layouts agree
+// (16-byte chunks need 16-byte aligned columns); element-wise copies transpose on the fly.
+// ---------------------------------------------------------------------------------------
+template <typename T, int BO, int BK, int NT, Layout SRC, Layout DST, int VEC, int PITCH>
+struct Stager {
+  static constexpr int ELEM = sizeof(T);
+
+  static __device__ __forceinline__ void load(T* __restrict__ s, const T* __restrict__ X0, int64_t ld, int o_valid,
+                                              int k_valid, int tid) {
+    if constexpr (SRC == DST) {
+      constexpr int CE = (SRC == OC) ? BO : BK;  // contiguous extent
+      constexpr int OE = (SRC == OC) ? BK : BO;  // number of lines
+      constexpr int CPL = CE / VEC;              // chunks per line
+      constexpr int TOTAL = OE * CPL;
+      constexpr int ITER = (TOTAL + NT - 1) / NT;
+      static_assert(CE % VEC == 0, "tile extent must be a multiple of the chunk");
+      const int c_valid = (SRC == OC) ? o_valid : k_valid;
+      const int l_valid = (SRC == OC) ? k_valid : o_valid;
+#pragma unroll
+      for (int it = 0; it < ITER; ++it) {
+        const int c = tid + it * NT;
+        if (TOTAL % NT != 0 && c >= TOTAL) break;
+        const int line = c / CPL;
+        const int cc = (c % CPL) * VEC;
+        int nvalid = c_valid - cc;
+        nvalid = nvalid < 0 ? 0 : (nvalid > VEC ? VEC : nvalid);
+        if (line >= l_valid) nvalid = 0;
+        const T* src = nvalid > 0 ? X0 + cc + (int64_t)line * ld : X0;
+        cp_async_zfill<VEC * ELEM>(s + line * PITCH + cc, src, nvalid * ELEM);
+      }
+    } else {
+      // element-wise transposing copy; runs of 8 along the source's contiguous dimension
+      constexpr int TOTAL = BO * BK;
+      constexpr int ITER = (TOTAL + NT - 1) / NT;
+      constexpr int RUN = 8;
+      static_assert(BK % RUN == 0 && BO % RUN == 0, "tile extents must be multiples of 8");
+#pragma unroll
+      for (int it = 0; it < ITER; ++it) {
+        const int c = tid + it * NT;
+        if (TOTAL % NT != 0 && c >= TOTAL) break;
+        int o, kk;
+        if constexpr (SRC == KC) {  // source k-contiguous
+          kk = (c % RUN) + RUN * (c / (RUN * BO));
+          o = (c / RUN) % BO;
+        } else {  // source o-contiguous
+          o = (c % RUN) + RUN * (c / (RUN * BK));
+          kk = (c / RUN) % BK;
+        }
+        const bool ok = (o < o_valid) && (kk < k_valid);
+        const T* src = X0;
+        if (ok) src = (SRC == KC) ? X0 + kk + (int64_t)o * ld : X0 + o + (int64_t)kk * ld;
+        T* dst = (DST == OC) ? s + kk * PITCH + o : s + o * PITCH + kk;
+        cp_async_zfill<ELEM>(dst, src, ok ? ELEM : 0);
+      }
+    }
+  }
+};
+
+// ---------------------------------------------------------------------------------------
+// Micro-kernel 1: FP64 tensor-core (DMMA) outer products, mma.sync m16n8k4.
+//
+// One warp owns a WTM x WTN block of the CTA tile as MI x NI fragments of 16 x 8; each
+// mma adds four rank-1 updates (k = 4) to a fragment.  All MI*NI mma of a k-step are
+// independent, as the paper's sizing rule asks.
+//
+// Fragment ownership (lane = 4*g + t, g = 0..7, t = 0..3), PTX m16n8k4 .f64:
+//   A (16x4): a0 = (row g, k t), a1 = (row g+8, k t);  B (4x8): b0 = (k t, col g);
+//   C (16x8): c0,c1 = (row g, cols 2t, 2t+1), c2,c3 = (row g+8, cols 2t, 2t+1).
+// The 16 fragment rows are mapped onto rows of C as  row r -> 2r (r < 8), 2(r-8)+1 (r >= 8),
+// so a lane's (a0, a1) are two adjacent rows (one 16-byte shared-memory load in the OC
+// layout) and (c0, c2) / (c1, c3) are adjacent rows of one column of C (one 16-byte store).
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ void dmma_m16n8k4(double (&c)[4], double a0, double a1, double b0) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k4.row.col.f64.f64.f64.f64 {%0,%1,%2,%3}, {%4,%5}, {%6}, {%0,%1,%2,%3};\n"
+      : "+d"(c[0]), "+d"(c[1]), "+d"(c[2]), "+d"(c[3])
+      : "d"(a0), "d"(a1), "d"(b0));
+}
+
+template <int BM_, int BN_, int BK_, int WARPS_M, int WARPS_N, bool TA, bool TB>
+struct DmmaMicro {
+  using T = double;
+  static constexpr int BM = BM_, BN = BN_, BK = BK_;
+  static constexpr int NT = 32 * WARPS_M * WARPS_N;
+  static constexpr int WTM = BM / WARPS_M, WTN = BN / WARPS_N;
+  static constexpr int MI = WTM / 16, NI = WTN / 8;
+  static_assert(WTM % 16 == 0 && WTN % 8 == 0 && BK % 16 == 0, "warp tile must be built from 16x8 fragments");
+  // Fragment loads read either layout, so tiles are staged in their source layout.
+  static constexpr Layout LA = TA ? KC : OC;
+  static constexpr Layout LB = TB ? OC : KC;
+  // Pitches (in doubles) that make every fragment load bank-conflict free:
+  //   OC: pitch = 4 (mod 16);  KC for A (rows 2g, 2g+1): pitch = 2 (mod 16);  KC for B: 4 (mod 16).
+  static constexpr int PA = (LA == OC) ? BM + 4 : BK + 2;
+  static constexpr int PB = (LB == OC) ? BN + 4 : BK + 4;
+  static constexpr int A_STAGE = (LA == OC) ? BK * PA : BM * PA;
+  static constexpr int B_STAGE = (LB == OC) ? BK * PB : BN * PB;
+  static constexpr int VEC = 2;
+
+  struct Acc {
+    double c[MI][NI][4];
+  };
+
+  static __device__ __forceinline__ void zero(Acc& acc) {
+#pragma unroll
+    for (int mi = 0; mi < MI; ++mi)
+#pragma unroll
+      for (int ni = 0; ni < NI; ++ni)
+#pragma unroll
+        for (int r = 0; r < 4; ++r) acc.c[mi][ni][r] = 0.0;
+  }
+
+  // One BK-deep slab: BK/4 k-steps of MI*NI independent mma.
+  static __device__ __forceinline__ void compute(Acc& acc, const double* __restrict__ sA,
+                                                 const double* __restrict__ sB, int warp_m, int warp_n, int lane) {
+    const int g = lane >> 2, t = lane & 3;
+    const int wm0 = warp_m * WTM, wn0 = warp_n * WTN;
+#pragma unroll
+    for (int ks = 0; ks < BK / 4; ++ks) {
+      const int kk = ks * 4 + t;
+      double a[MI][2], b[NI];
+#pragma unroll
+      for (int mi = 0; mi < MI; ++mi) {
+        const int r = wm0 + mi * 16 + 2 * g;
+        if constexpr (LA == OC) {
+          const double2 v = *reinterpret_cast<const double2*>(sA + kk * PA + r);
+          a[mi][0] = v.x;
+          a[mi][1] = v.y;
+        } else {
+          a[mi][0] = sA[r * PA + kk];
+          a[mi][1] = sA[(r + 1) * PA + kk];
+        }
+      }
+#pragma unroll
+      for (int ni = 0; ni < NI; ++ni) {
+        const int cidx = wn0 + ni * 8 + g;
+        b[ni] = (LB == OC) ? sB[kk * PB + cidx] : sB[cidx * PB + kk];
+      }
+#pragma unroll
+      for (int mi = 0; mi < MI; ++mi)
+#pragma unroll
+        for (int ni = 0; ni < NI; ++ni) dmma_m16n8k4(acc.c[mi][ni], a[mi][0], a[mi][1], b[ni]);
+    }
+  }
+
+  // C := alpha*acc + beta*C on the warp's block; rows >= m and columns >= n are skipped.
+  static __device__ __forceinline__ void epilogue(const Acc& acc, const GemmArgs<double>& p, int64_t m0, int64_t n0,
+                                                  int warp_m, int warp_n, int lane) {
+    const int g = lane >> 2, t = lane & 3;
+    const bool vec_ok = ((reinterpret_cast<uintptr_t>(p.C) & 15) == 0) && ((p.ldc & 1) == 0);
+    const bool use_beta = (p.beta != 0.0);
+#pragma unroll
+    for (int ni = 0; ni < NI; ++ni) {
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const int64_t col = n0 + warp_n * WTN + ni * 8 + 2 * t + h;
+        if (col >= p.n) continue;
+        double* ccol = p.C + col * p.ldc;
+#pragma unroll
+        for (int mi = 0; mi < MI; ++mi) {
+          const int64_t row = m0 + warp_m * WTM + mi * 16 + 2 * g;
+          if (row >= p.m) continue;
+          double v0 = p.alpha * acc.c[mi][ni][h], v1 = p.alpha * acc.c[mi][ni][2 + h];
+          double* dst = ccol + row;
+          if (vec_ok && row + 1 < p.m) {
+            if (use_beta) {
+              const double2 old = *reinterpret_cast<const double2*>(dst);
+              v0 += p.beta * old.x;
+              v1 += p.beta * old.y;
+            }
+            *reinterpret_cast<double2*>(dst) = make_double2(v0, v1);
+          } else {
+            if (use_beta) v0 += p.beta * dst[0];
+            dst[0] = v0;
+            if (row + 1 < p.m) {
+              if (use_beta) v1 += p.beta * dst[1];
+              dst[1] = v1;
+            }
+          }
+        }
+      }
+    }
+  }
+};
+
+// ---------------------------------------------------------------------------------------
+// Micro-kernel 2: scalar FMA outer products (FP32 FFMA; also FP64 DFMA).
+//
+// Both operands are packed into the OC layout (the paper's packed micro-panels: a column of
+// A and a row of B are each contiguous), transposing while staging when the source is
+// k-contiguous.  Each thread keeps a TM x TN = 8 x 8 accumulator block in registers and per
+// k performs the rank-1 update acc += a b^T with a (8 values) and b (8 values) fetched by
+// 16-byte shared-memory loads: 64 independent FMAs per outer product.
+// A warp is 8 lanes along m by 4 lanes along n, so it covers 64 x 32 of C.
+// ---------------------------------------------------------------------------------------
+template <typename T_, int BM_, int BN_, int BK_, int WARPS_M, int WARPS_N, bool TA, bool TB>
+struct SimtMicro {
+  using T = T_;
+  static constexpr int BM = BM_, BN = BN_, BK = BK_;
+  static constexpr int NT = 32 * WARPS_M * WARPS_N;
+  static constexpr int VEC = 16 / sizeof(T);
+  static constexpr int TM = 8, TN = 8;
+  static constexpr int WTM = 8 * TM, WTN = 4 * TN;
+  static_assert(BM == WARPS_M * WTM && BN == WARPS_N * WTN, "CTA tile must be warps x (64 x 32)");
+  static constexpr Layout LA = OC, LB = OC;
+  static constexpr int PA = BM + VEC, PB = BN + VEC;
+  static constexpr int A_STAGE = BK * PA, B_STAGE = BK * PB;
+  using VT = typename std::conditional<sizeof(T) == 4, float4, double2>::type;
+
+  struct Acc {
+    T c[TM][TN];
+  };
+
+  static __device__ __forceinline__ void zero(Acc& acc) {
+#pragma unroll
+    for (int i = 0; i < TM; ++i)
+#pragma unroll
+      for (int j = 0; j < TN; ++j) acc.c[i][j] = T(0);
+  }
+
+  static __device__ __forceinline__ void load_vec(T* dst, const T* src) {
+    const VT v = *reinterpret_cast<const VT*>(src);
+    if constexpr (sizeof(T) == 4) {
+      dst[0] = v.x, dst[1] = v.y, dst[2] = v.z, dst[3] = v.w;
+    } else {
+      dst[0] = v.x, dst[1] = v.y;
+    }
+  }
+
+  static __device__ __forceinline__ void compute(Acc& acc, const T* __restrict__ sA, const T* __restrict__ sB,
+                                                 int warp_m, int warp_n, int lane) {
+    const int lx = lane & 7, ly = lane >> 3;
+    const T* pa = sA + warp_m * WTM + lx * VEC;
+    const T* pb = sB + warp_n * WTN + ly * VEC;
+#pragma unroll
+    for (int kk = 0; kk < BK; ++kk) {
+      T a[TM], b[TN];
+#pragma unroll
+      for (int gi = 0; gi < TM / VEC; ++gi) load_vec(a + gi * VEC, pa + kk * PA + gi * 8 * VEC);
+#pragma unroll
+      for (int gj = 0; gj < TN / VEC; ++gj) load_vec(b + gj * VEC, pb + kk * PB + gj * 4 * VEC);
+#pragma unroll
+      for (int i = 0; i < TM; ++i)
+#pragma unroll
+        for (int j = 0; j < TN; ++j) acc.c[i][j] = fma(a[i], b[j], acc.c[i][j]);
+    }
+  }
+
+  static __device__ __forceinline__ void epilogue(const Acc& acc, const GemmArgs<T>& p, int64_t m0, int64_t n0,
+                                                  int warp_m, int warp_n, int lane) {
+    const int lx = lane & 7, ly = lane >> 3;
+    const bool vec_ok = ((reinterpret_cast<uintptr_t>(p.C) & 15) == 0) && ((p.ldc % VEC) == 0);
+    const bool use_beta = (p.beta != T(0));
+#pragma unroll
+    for (int j = 0; j < TN; ++j) {
+      const int64_t col = n0 + warp_n * WTN + (j / VEC) * 4 * VEC + ly * VEC + (j % VEC);
+      if (col >= p.n) continue;
+      T* ccol = p.C + col * p.ldc;
+#pragma unroll
+      for (int gi = 0; gi < TM / VEC; ++gi) {
+        const int64_t row = m0 + warp_m * WTM + gi * 8 * VEC + lx * VEC;
+        if (row >= p.m) continue;
+        T v[VEC];
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) v[e] = p.alpha * acc.c[gi * VEC + e][j];
+        T* dst = ccol + row;
+        if (vec_ok && row + VEC <= p.m) {
+          if (use_beta) {
+            T old[VEC];
+            load_vec(old, dst);
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) v[e] += p.beta * old[e];
+          }
+          VT out;
+          if constexpr (sizeof(T) == 4) {
+            out = make_float4(v[0], v[1], v[2], v[3]);
+          } else {
+            out = make_double2(v[0], v[1]);
+          }
+          *reinterpret_cast<VT*>(dst) = out;
+        } else {
+#pragma unroll
+          for (int e = 0; e < VEC; ++e) {
+            if (row + e < p.m) {
+              if (use_beta) v[e] += p.beta * dst[e];
+              dst[e] = v[e];
+            }
+          }
+        }
+      }
+    }
+  }
+};
+
+// ---------------------------------------------------------------------------------------
+// The kernel.  One CTA computes one BM x BN tile of C.
+//   ALIGNED: every column of A and B starts on a 16-byte boundary (base pointers 16-byte
+//   aligned, leading dimensions multiples of 16/sizeof(T)); otherwise operands are staged
+//   element by element.
+// ---------------------------------------------------------------------------------------
+template <class Micro, int STAGES, bool TA, bool TB, bool ALIGNED>
+struct GemmKernel {
+  using T = typename Micro::T;
+  static constexpr int BM = Micro::BM, BN = Micro::BN, BK = Micro::BK, NT = Micro::NT;
+  static constexpr Layout SRC_A = TA ? KC : OC;
+  static constexpr Layout SRC_B = TB ? OC : KC;
+  static constexpr int VEC = ALIGNED ? (16 / (int)sizeof(T)) : 1;
+  using StageA = Stager<T, BM, BK, NT, SRC_A, Micro::LA, VEC, Micro::PA>;
+  using StageB = Stager<T, BN, BK, NT, SRC_B, Micro::LB, VEC, Micro::PB>;
+  static constexpr size_t SMEM_BYTES = (size_t)STAGES * (Micro::A_STAGE + Micro::B_STAGE) * sizeof(T);
+
+  static __device__ __forceinline__ void run(const GemmArgs<T>& p) {
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    T* sA = reinterpret_cast<T*>(smem_raw);
+    T* sB = sA + STAGES * Micro::A_STAGE;
+
+    const int tid = threadIdx.x;
+    const int warp = tid >> 5, lane = tid & 31;
+    const int warp_m = warp % (BM / Micro::WTM), warp_n = warp / (BM / Micro::WTM);
+
+    int tm, tn;
+    tile_coords(blockIdx.x, p.tiles_m, p.tiles_n, p.group_m, tm, tn);
+    const int64_t m0 = (int64_t)tm * BM, n0 = (int64_t)tn * BN;
+    const int m_valid = (int)min((int64_t)BM, p.m - m0), n_valid = (int)min((int64_t)BN, p.n - n0);
+
+    // element (m0, 0) of op(A) and (0, n0) of op(B)
+    const T* gA = TA ? p.A + m0 * p.lda : p.A + m0;
+    const T* gB = TB ? p.B + n0 : p.B + n0 * p.ldb;
+    const int64_t stepA = TA ? (int64_t)BK : (int64_t)BK * p.lda;  // advance by BK along k
+    const int64_t stepB = TB ? (int64_t)BK * p.ldb : (int64_t)BK;
+
+    const int KT = (int)((p.k + BK - 1) / BK);
+
+    auto stage = [&](int kt) {
+      const int slot = kt % STAGES;
+      const int k_valid = (int)min((int64_t)BK, p.k - (int64_t)kt * BK);
+      StageA::load(sA + slot * Micro::A_STAGE, gA + kt * stepA, p.lda, m_valid, k_valid, tid);
+      StageB::load(sB + slot * Micro::B_STAGE, gB + kt * stepB, p.ldb, n_valid, k_valid, tid);
+    };
+
+    // ramp-up: fill STAGES-1 slots (the first of the paper's three stages of the k-loop)
+#pragma unroll
+    for (int s = 0; s < STAGES - 1; ++s) {
+      if (s < KT) stage(s);
+      cp_async_commit();
+    }
+
+    typename Micro::Acc acc;
+    Micro::zero(acc);
+
+    // steady state: wait for slab kt, refill the slot freed in the previous iteration, compute
+    for (int kt = 0; kt < KT; ++kt) {
+      cp_async_wait<STAGES - 2>();
+      __syncthreads();
+      const int next = kt + STAGES - 1;
+      if (next < KT) stage(next);
+      cp_async_commit();
+      const int slot = kt % STAGES;
+      Micro::compute(acc, sA + slot * Micro::A_STAGE, sB + slot * Micro::B_STAGE, warp_m, warp_n, lane);
+    }
+    cp_async_wait<0>();
+
+    // drain: fused alpha/beta epilogue
+    Micro::epilogue(acc, p, m0, n0, warp_m, warp_n, lane);
+  }
+};
+
+template <class Kernel, int MIN_CTAS>
+__global__ void __launch_bounds__(Kernel::NT, MIN_CTAS) gemm_kernel(const GemmArgs<typename Kernel::T> p) {
+  Kernel::run(p);
+}
+
+// C := beta*C for the quick-return cases (alpha == 0 or k == 0); beta == 0 stores zeros
+// without reading C.
+template <typename T>
+__global__ void scale_kernel(int64_t m, int64_t n, T beta, T* C, int64_t ldc) {
+  const int64_t total = m * n;
+  for (int64_t idx = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; idx < total;
+       idx += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t i = idx % m, j = idx / m;
+    T* c = C + i + j * ldc;
+    *c = (beta == T(0)) ? T(0) : beta * *c;
+  }
+}
+
+}  // namespace b2

@@ -1,0 +1,71 @@
+// Host-side launch of one kernel variant: picks the (transA, transB, aligned) instantiation,
+// raises the dynamic shared-memory limit once per device and launches on the caller's stream.
+#pragma once
+#include "b2gemm.h"
+#include "gemm_kernel.cuh"
+
+namespace b2 {
+
+// Static description of a variant, used by the selector and by b2_gemm_query_config.
+struct VariantInfo {
+  const char* name;
+  const char* micro;  // "dmma" | "dfma" | "ffma"
+  int bm, bn, bk, stages, threads, ctas_per_sm;
+};
+
+template <typename T>
+using LaunchFn = int (*)(const GemmArgs<T>& args, bool ta, bool tb, bool aligned, cudaStream_t stream);
+
+template <class Kernel, int MIN_CTAS>
+int launch_one(const GemmArgs<typename Kernel::T>& args, cudaStream_t stream) {
+  static bool configured[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return B2_ERR_LAUNCH;
+  auto kfn = gemm_kernel<Kernel, MIN_CTAS>;
+  if (dev < 0 || dev >= 64 || !configured[dev]) {
+    if (cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Kernel::SMEM_BYTES) !=
+        cudaSuccess)
+      return B2_ERR_LAUNCH;
+    if (dev >= 0 && dev < 64) configured[dev] = true;
+  }
+  const long long tiles = (long long)args.tiles_m * args.tiles_n;
+  if (tiles <= 0 || tiles > 0x7fffffffLL) return B2_ERR_LAUNCH;
+  kfn<<<(unsigned)tiles, Kernel::NT, Kernel::SMEM_BYTES, stream>>>(args);
+  return cudaGetLastError() == cudaSuccess ? B2_OK : B2_ERR_LAUNCH;
+}
+
+// MicroT<TA, TB> is the micro-kernel policy for a transpose combination.
+template <template <bool, bool> class MicroT, int STAGES, int MIN_CTAS>
+struct VariantLauncher {
+  template <bool TA, bool TB>
+  using Micro = MicroT<TA, TB>;
+  using T = typename MicroT<false, false>::T;
+
+  template <bool TA, bool TB>
+  static int pick_aligned(const GemmArgs<T>& a, bool aligned, cudaStream_t s) {
+    if (aligned) return launch_one<GemmKernel<MicroT<TA, TB>, STAGES, TA, TB, true>, MIN_CTAS>(a, s);
+    return launch_one<GemmKernel<MicroT<TA, TB>, STAGES, TA, TB, false>, MIN_CTAS>(a, s);
+  }
+
+  static int launch(const GemmArgs<T>& args_in, bool ta, bool tb, bool aligned, cudaStream_t s) {
+    GemmArgs<T> a = args_in;
+    constexpr int BM = MicroT<false, false>::BM, BN = MicroT<false, false>::BN;
+    a.tiles_m = (int)((a.m + BM - 1) / BM);
+    a.tiles_n = (int)((a.n + BN - 1) / BN);
+    if (a.group_m <= 0) a.group_m = 8;
+    if (!ta && !tb) return pick_aligned<false, false>(a, aligned, s);
+    if (!ta && tb) return pick_aligned<false, true>(a, aligned, s);
+    if (ta && !tb) return pick_aligned<true, false>(a, aligned, s);
+    return pick_aligned<true, true>(a, aligned, s);
+  }
+};
+
+// Variant tables, defined in gemm_f64_*.cu / gemm_f32_*.cu
+int f64_variant_count();
+const VariantInfo& f64_variant_info(int v);
+LaunchFn<double> f64_variant_launch(int v);
+int f32_variant_count();
+const VariantInfo& f32_variant_info(int v);
+LaunchFn<float> f32_variant_launch(int v);
+
+}  // namespace b2

@@ -1,0 +1,78 @@
+// Analytic choice of the CTA tile (host code, no CUDA).
+//
+// The paper picks a micro-kernel by estimating, per candidate, the time its instruction mix
+// needs to clear the slowest pipeline (Section 4, "Little's Law": throughput = min over
+// pipelines of rate / jobs) and keeps the best.  The same idea one level up: for each
+// candidate CTA tile, estimate the clocks one SM needs for its share of the tiles from the
+// three "pipelines" a tile occupies -- the arithmetic pipe, the L2->shared-memory feed and the
+// C traffic of the epilogue -- and keep the candidate with the smallest estimate.
+#pragma once
+#include <stdint.h>
+
+namespace b2 {
+
+struct TileChoice {
+  int bm, bn, bk;
+  int threads;
+  int ctas_per_sm;   // CTAs of this variant that fit on one SM
+  bool explicit_only;  // never chosen automatically (comparison variants)
+};
+
+// Measured / derived machine rates per SM (B200): FP64 and FP32 multiply-adds per clock, the
+// L2->SM feed and the SM's share of HBM bandwidth in bytes per clock, and fixed per-tile costs.
+struct MachineRates {
+  double fma_per_clk;        // 64 (fp64: DFMA and DMMA alike), 128 (fp32 FFMA)
+  double l2_bytes_per_clk;   // sustainable L2 -> shared-memory feed per SM
+  double hbm_bytes_per_clk;  // HBM bytes per clock per SM (6.5 TB/s / 148 SMs / 1.965 GHz)
+  double tile_fixed_clks;    // launch + pipeline ramp-up + drain of one CTA
+};
+
+inline MachineRates machine_rates(int elem_bytes) {
+  MachineRates r;
+  r.fma_per_clk = elem_bytes == 8 ? 64.0 : 128.0;
+  r.l2_bytes_per_clk = 24.0;
+  r.hbm_bytes_per_clk = 22.0;
+  r.tile_fixed_clks = 4000.0;
+  return r;
+}
+
+// Estimated clocks for one SM to finish its share of the problem with tile `c`.
+inline double estimate_clks(const TileChoice& c, int64_t m, int64_t n, int64_t k, int sms, int elem_bytes) {
+  const MachineRates r = machine_rates(elem_bytes);
+  const double tiles = (double)((m + c.bm - 1) / c.bm) * (double)((n + c.bn - 1) / c.bn);
+  const double kt = (double)((k + c.bk - 1) / c.bk);
+  // tiles are handed out CTA by CTA; an SM ends up with ceil(tiles / sms) of them
+  const double per_sm = (double)(int64_t)((tiles + sms - 1) / sms);
+  const double fma_tile = (double)c.bm * c.bn * c.bk * kt;
+  // arithmetic pipe
+  double t_math = fma_tile / r.fma_per_clk;
+  // feed: bytes of A and B a tile pulls through L2 per multiply-add
+  const double feed_tile = (double)(c.bm + c.bn) * c.bk * kt * elem_bytes;
+  const double t_feed = feed_tile / r.l2_bytes_per_clk;
+  const double t_main = t_math > t_feed ? t_math : t_feed;
+  // epilogue: C read + write at the SM's share of HBM bandwidth
+  const double t_epi = 2.0 * c.bm * c.bn * elem_bytes / r.hbm_bytes_per_clk;
+  const double t_fixed = r.tile_fixed_clks + t_epi;
+  // With >= 2 resident CTAs one tile's ramp-up/epilogue overlaps another tile's main loop;
+  // with a single resident CTA every tile pays it.
+  const double resident = per_sm < c.ctas_per_sm ? per_sm : c.ctas_per_sm;
+  if (resident >= 2.0) {
+    const double overlapped = per_sm * (t_main > t_epi ? t_main : t_epi);
+    return overlapped + t_fixed;
+  }
+  return per_sm * (t_main + t_fixed);
+}
+
+// Index of the candidate with the smallest estimate.
+inline int select_tile(const TileChoice* cand, int count, int64_t m, int64_t n, int64_t k, int sms, int elem_bytes) {
+  int best = -1;
+  double best_t = 0.0;
+  for (int i = 0; i < count; ++i) {
+    if (cand[i].explicit_only) continue;
+    const double t = estimate_clks(cand[i], m, n, k, sms, elem_bytes);
+    if (best < 0 || t < best_t) best = i, best_t = t;
+  }
+  return best < 0 ? 0 : best;
+}
+
+}  // namespace b2
