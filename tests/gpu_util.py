@@ -1,0 +1,92 @@
+"""Shared machinery of the GPU parity tests: run one problem through the C-ABI and through the oracle on the
+same seeded inputs and compare element by element (all of C, or a column sample for big problems)."""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from helpers import U
+from paper_1611_08035_b200 import synth
+
+TORCH_DT = {"d": torch.float64, "s": torch.float32, "z": torch.complex128}
+
+
+def sample_columns(n: int, tile: int = 64, extra: int = 24, seed: int = 0):
+    """First, last, both sides of every `tile` boundary hit by a coarse stride, plus seeded random columns."""
+    cols = {0, n - 1}
+    for b in range(tile, n, max(tile, (n // 8) // tile * tile)):
+        cols.update({b - 1, b})
+    rng = np.random.default_rng(seed)
+    cols.update(int(c) for c in rng.integers(0, n, size=extra))
+    return sorted(c for c in cols if 0 <= c < n)
+
+
+def run_and_check(b2, oracle, kind, transa, transb, m, n, k, alpha, beta, dist="uniform", seed=0, pad=False,
+                  variant=None, cols=None, c_dist=None, expect_exact=False, lds=None, offset=0, factor=None):
+    """Returns the largest observed error/bound ratio.  kind: 'd', 's' (real) or 'z' (4M complex).
+
+    Checks: every compared element within 2*k*u*S (complex: 2*(2k+4)*u*S per component); bit-exact when
+    expect_exact; padding rows of C and unsampled nothing-else untouched; A and B unchanged.
+    `offset` shifts every base pointer by that many elements (misaligned bases)."""
+    tdt = TORCH_DT[kind]
+    (ra, ca), (rb, cb) = synth.operand_shapes(transa, transb, m, n, k)
+    if lds is not None:
+        lda, ldb, ldc = lds
+    elif pad:
+        lda, ldb, ldc = synth.padded_ld(ra), synth.padded_ld(rb), synth.padded_ld(m)
+    else:
+        lda = ldb = ldc = None
+    A, lda, B, ldb, C, ldc = synth.gemm_inputs(transa, transb, m, n, k, dist, seed, tdt, lda, ldb, ldc, c_dist=c_dist)
+    An, Bn, Cn = A.numpy(), B.numpy(), C.numpy()
+
+    def dev(x):
+        if offset:
+            buf = torch.empty(x.numel() + offset, dtype=x.dtype, device="cuda")
+            buf[offset:].copy_(x)
+            return buf, buf[offset:]
+        d = x.cuda()
+        return d, d
+
+    Ah, Ad = dev(A)
+    Bh, Bd = dev(B)
+    Ch, Cd = dev(C)
+    if kind == "z":
+        ws = torch.empty(max(256, b2.b2_zgemm4m_workspace_bytes(transa, transb, m, n, k)), dtype=torch.uint8,
+                         device="cuda")
+        b2.b2_zgemm4m(transa, transb, m, n, k, alpha, Ad, lda, Bd, ldb, beta, Cd, ldc, ws)
+    else:
+        fn = b2.b2_dgemm if kind == "d" else b2.b2_sgemm
+        fn(transa, transb, m, n, k, alpha, Ad, lda, Bd, ldb, beta, Cd, ldc, variant=variant)
+    torch.cuda.synchronize()
+    got = Cd.cpu().numpy()
+    assert torch.equal(Ad.cpu().view(torch.uint8), A.view(torch.uint8)), "A was modified"
+    assert torch.equal(Bd.cpu().view(torch.uint8), B.view(torch.uint8)), "B was modified"
+
+    want = Cn.copy()
+    oracle.ref_gemm(transa, transb, m, n, k, alpha, An, lda, Bn, ldb, beta, want, ldc, cols=cols)
+    _, S = oracle.ref_gemm_hi(transa, transb, m, n, k, alpha, An, lda, Bn, ldb, beta, Cn, ldc, cols=cols)
+    if m == 0 or n == 0:
+        assert got.tobytes() == Cn.tobytes()
+        return 0.0
+    sel = list(range(n)) if cols is None else list(cols)
+    G = got.reshape(n, ldc)
+    W = want.reshape(n, ldc)
+    # padding rows of every column, and (for the GPU, which computes all columns) nothing outside m x n
+    assert G[:, m:].tobytes() == Cn.reshape(n, ldc)[:, m:].tobytes(), "padding rows of C were written"
+    g, w = G[sel, :m], W[sel, :m]
+    Sv = S.reshape(n, max(1, m))[sel, :m]
+    if expect_exact:
+        assert g.tobytes() == w.tobytes(), "integer-valued problem is not bit-exact"
+        return 0.0
+    u = U[np.dtype(Cn.dtype)]
+    if kind == "z":
+        bound = 2.0 * (2 * k + 4) * u * Sv
+        err = np.maximum(np.abs(g.real - w.real), np.abs(g.imag - w.imag))
+    else:
+        bound = (2.0 * k * u if factor is None else factor) * Sv
+        err = np.abs(g.astype(np.float64) - w.astype(np.float64))
+    assert np.all(np.isfinite(g.view(np.float64) if kind == "z" else g)), "non-finite result"
+    bad = err > bound
+    assert not bad.any(), f"{int(bad.sum())} elements exceed the bound; worst ratio " \
+                          f"{float((err / np.maximum(bound, 1e-300)).max()):.3g}"
+    return float((err / np.maximum(bound, 1e-300)).max())

@@ -1,0 +1,266 @@
+"""GPU parity tests: the CUDA path, called through the C-ABI, against the CPU oracle on identical seeded inputs.
+
+Tolerances (written here on purpose): integer-valued problems must be bit-exact; otherwise every element must
+satisfy |C - C_ref| <= 2*k*u*(|alpha||A||B| + |beta||C|)_ij with u = 2^-53 (fp64) or 2^-24 (fp32); the 4M complex
+entry uses 2*(2k+4)*u per component (each component is a 2k-term sum of products of a once-rounded alpha*A).
+"""
+import itertools
+
+import numpy as np
+import pytest
+import torch
+
+from gpu_util import run_and_check, sample_columns
+from paper_1611_08035_b200 import synth
+
+pytestmark = pytest.mark.gpu
+TRANS = list(itertools.product("NT", "NT"))
+
+
+def nvariants(b2, kind):
+    return b2.b2_variant_count(0 if kind == "d" else 1)
+
+
+# ---- the five benchmark configurations -------------------------------------------------------------
+
+def test_config1_dgemm_256(b2, oracle):
+    r = run_and_check(b2, oracle, "d", "N", "N", 256, 256, 256, 1.0, 0.0, dist="uniform", seed=0, c_dist="zero")
+    assert r <= 1.0
+
+
+@pytest.mark.parametrize("kind", ["d", "s"])
+@pytest.mark.parametrize("size", [512, 1024])
+def test_config2_square_small_full(b2, oracle, kind, size):
+    seed = (2000 if kind == "d" else 2100) + int(np.log2(size))
+    run_and_check(b2, oracle, kind, "N", "N", size, size, size, 1.5, 0.5, dist="uniform", seed=seed)
+    run_and_check(b2, oracle, kind, "N", "N", size, size, size, 1.5, 0.5, dist="int9", seed=seed, expect_exact=True)
+
+
+@pytest.mark.parametrize("kind", ["d", "s"])
+@pytest.mark.parametrize("size", [2048, 4096, 8192])
+def test_config2_square_large_sampled(b2, oracle, kind, size):
+    """Full benchmark sizes in the launch configuration the benchmark times (automatic variant, aligned
+    operands); the oracle evaluates a column sample (first, last, tile boundaries, random)."""
+    seed = (2000 if kind == "d" else 2100) + int(np.log2(size))
+    cols = sample_columns(size, tile=64, extra=16 if size == 8192 else 24, seed=seed)
+    run_and_check(b2, oracle, kind, "N", "N", size, size, size, 1.5, 0.5, dist="uniform", seed=seed, cols=cols)
+    if size <= 4096:
+        run_and_check(b2, oracle, kind, "N", "N", size, size, size, 1.5, 0.5, dist="int9", seed=seed, cols=cols,
+                      expect_exact=True)
+
+
+def test_config2_integer_8192_fp64_sampled(b2, oracle):
+    cols = sample_columns(8192, tile=64, extra=8, seed=1)
+    run_and_check(b2, oracle, "d", "N", "N", 8192, 8192, 8192, 1.5, 0.5, dist="int9", seed=2013, cols=cols,
+                  expect_exact=True)
+
+
+@pytest.mark.parametrize("k", [64, 128, 256])
+def test_config3_rank_k_update_sampled(b2, oracle, k):
+    cols = sample_columns(16384, tile=64, extra=40, seed=k)
+    run_and_check(b2, oracle, "d", "N", "N", 16384, 16384, k, -1.0, 1.0, dist="normal", seed=3000 + k, cols=cols)
+
+
+@pytest.mark.parametrize("kind", ["d", "s"])
+@pytest.mark.parametrize("ta,tb", TRANS)
+def test_config4_fringe_and_transposes(b2, oracle, kind, ta, tb):
+    seed = 4000 + 2 * (ta == "T") + (tb == "T")
+    run_and_check(b2, oracle, kind, ta, tb, 1001, 999, 1003, 0.7, -0.3, dist="uniform", seed=seed, pad=True)
+    run_and_check(b2, oracle, kind, ta, tb, 1001, 999, 1003, 1.5, 0.5, dist="int9", seed=seed, pad=True,
+                  expect_exact=True)
+
+
+def test_config5_complex_4m_4096_sampled(b2, oracle):
+    cols = sample_columns(4096, tile=64, extra=8, seed=5)
+    run_and_check(b2, oracle, "z", "N", "N", 4096, 4096, 4096, 1 + 0.5j, 0j, dist="uniform", seed=5000, cols=cols)
+
+
+# ---- every variant, every transpose, shapes around every tile edge ---------------------------------
+
+EDGE = [1, 2, 3, 7, 8, 9, 15, 16, 17, 31, 33, 63, 64, 65, 127, 128, 129, 191, 257]
+
+
+@pytest.mark.parametrize("kind", ["d", "s"])
+def test_all_variants_edge_shapes(b2, oracle, kind):
+    rng = np.random.default_rng(42)
+    for v in range(nvariants(b2, kind)):
+        for ta, tb in TRANS:
+            for trial in range(10):
+                m, n, k = (int(rng.choice(EDGE)) for _ in range(3))
+                pad = bool(trial % 2)
+                run_and_check(b2, oracle, kind, ta, tb, m, n, k, 0.7, -0.3, seed=trial, pad=pad, variant=v)
+                run_and_check(b2, oracle, kind, ta, tb, m, n, k, 1.5, 0.5, dist="int9", seed=trial, pad=pad,
+                              variant=v, expect_exact=True)
+
+
+@pytest.mark.parametrize("kind", ["d", "s"])
+def test_all_variants_multi_tile_ragged(b2, oracle, kind):
+    """Several tiles in both directions with ragged tails in m, n and k, aligned and padded leading dimensions,
+    beta == 0 and beta != 0."""
+    for v in range(nvariants(b2, kind)):
+        for ta, tb in TRANS:
+            run_and_check(b2, oracle, kind, ta, tb, 333, 270, 145, 0.7, -0.3, seed=v, pad=True, variant=v)
+            run_and_check(b2, oracle, kind, ta, tb, 300, 260, 136, 1.0, 0.0, seed=v, pad=False, variant=v)
+            run_and_check(b2, oracle, kind, ta, tb, 300, 260, 136, 1.5, 0.5, dist="int9", seed=v, variant=v,
+                          expect_exact=True)
+
+
+@pytest.mark.parametrize("kind", ["d", "s"])
+def test_misaligned_base_pointers(b2, oracle, kind):
+    """Base pointers shifted by one element (8- or 4-byte aligned only) with otherwise aligned leading dimensions."""
+    for ta, tb in TRANS:
+        run_and_check(b2, oracle, kind, ta, tb, 200, 136, 75, 0.7, -0.3, seed=3, offset=1)
+        run_and_check(b2, oracle, kind, ta, tb, 200, 136, 75, 1.5, 0.5, dist="int9", seed=3, offset=1, expect_exact=True)
+
+
+def test_skinny_and_degenerate_shapes(b2, oracle):
+    for kind in "ds":
+        for (m, n, k) in [(1, 1, 1), (1, 1000, 1), (1000, 1, 1), (1, 1, 1000), (5, 3, 0), (0, 7, 9), (7, 0, 9),
+                          (2049, 3, 5), (3, 2049, 5), (64, 64, 4097)]:
+            for ta, tb in TRANS:
+                run_and_check(b2, oracle, kind, ta, tb, m, n, k, 0.7, -0.3, seed=m + n + k, pad=True)
+
+
+# ---- BLAS conventions ------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("kind", ["d", "s"])
+def test_quick_returns_and_nan_poison(b2, oracle, kind):
+    tdt = torch.float64 if kind == "d" else torch.float32
+    fn = b2.b2_dgemm if kind == "d" else b2.b2_sgemm
+    m, n, k = 70, 50, 40
+    A, lda, B, ldb, C, ldc = synth.gemm_inputs("N", "N", m, n, k, "uniform", 9, tdt, m + 3, k + 3, m + 3)
+    nanA, nanB = torch.full_like(A, float("nan")).cuda(), torch.full_like(B, float("nan")).cuda()
+    Cv = C.view(n, ldc)
+    # beta == 0: NaN in the old C must not propagate
+    Cd = torch.full_like(C, float("nan")).cuda()
+    fn("N", "N", m, n, k, 1.0, A.cuda(), lda, B.cuda(), ldb, 0.0, Cd, ldc)
+    out = Cd.cpu().view(n, ldc)
+    assert torch.isfinite(out[:, :m]).all() and torch.isnan(out[:, m:]).all()
+    # alpha == 0: A, B not referenced (NaN-filled); C = beta*C exactly
+    Cd = C.cuda()
+    fn("N", "N", m, n, k, 0.0, nanA, lda, nanB, ldb, 0.5, Cd, ldc)
+    out = Cd.cpu().view(n, ldc)
+    assert torch.equal(out[:, :m], 0.5 * Cv[:, :m]) and torch.equal(out[:, m:], Cv[:, m:])
+    # alpha == 0 and beta == 0: zeros
+    Cd = torch.full_like(C, float("nan")).cuda()
+    fn("N", "N", m, n, k, 0.0, nanA, lda, nanB, ldb, 0.0, Cd, ldc)
+    assert (Cd.cpu().view(n, ldc)[:, :m] == 0).all()
+    # k == 0 with null A and B: C = beta*C
+    Cd = C.cuda()
+    fn("N", "N", m, n, 0, 1.0, None, max(1, m), None, 1, -1.0, Cd, ldc)
+    assert torch.equal(Cd.cpu().view(n, ldc)[:, :m], -Cv[:, :m])
+    # alpha == 0, beta == 1 / empty problems: untouched
+    Cd = C.cuda()
+    fn("N", "N", m, n, k, 0.0, nanA, lda, nanB, ldb, 1.0, Cd, ldc)
+    fn("N", "N", 0, n, k, 1.0, None, 1, B.cuda(), ldb, 0.0, Cd, ldc)
+    fn("N", "N", m, 0, k, 1.0, A.cuda(), lda, None, ldb, 0.0, Cd, ldc)
+    torch.cuda.synchronize()
+    assert torch.equal(Cd.cpu().view(torch.uint8), C.view(torch.uint8))
+    # NaN in A propagates to its row of C even when B is zero (no shortcuts on zeros)
+    A2 = A.clone()
+    A2.view(k, lda)[1, 2] = float("nan")
+    Cd = torch.zeros_like(C).cuda()
+    fn("N", "N", m, n, k, 1.0, A2.cuda(), lda, torch.zeros_like(B).cuda(), ldb, 0.0, Cd, ldc)
+    out = Cd.cpu().view(n, ldc)
+    assert torch.isnan(out[:, 2]).all() and (out[:, [0, 1, 3]] == 0).all()
+
+
+def test_lowercase_and_c_transposes(b2, oracle):
+    for kind in "ds":
+        run_and_check(b2, oracle, kind, "n", "t", 65, 33, 17, 0.7, -0.3, seed=1)
+        run_and_check(b2, oracle, kind, "c", "n", 65, 33, 17, 0.7, -0.3, seed=1)
+        run_and_check(b2, oracle, kind, "C", "c", 65, 33, 17, 0.7, -0.3, seed=1)
+
+
+def test_runtime_argument_errors_launch_nothing(b2):
+    C = torch.ones(64, dtype=torch.float64, device="cuda")
+    A = torch.ones(64, dtype=torch.float64, device="cuda")
+    assert b2.b2_dgemm("N", "N", 4, 4, 4, 1.0, None, 4, A, 4, 0.0, C, 4, check=False) == -7
+    assert b2.b2_dgemm("N", "N", 4, 4, 4, 1.0, A, 4, None, 4, 0.0, C, 4, check=False) == -9
+    assert b2.b2_dgemm("N", "N", 4, 4, 4, 1.0, A, 4, A, 4, 0.0, None, 4, check=False) == -12
+    assert b2.b2_dgemm("N", "N", 4, 4, 4, 1.0, A, 3, A, 4, 0.0, C, 4, check=False) == -8
+    assert b2.b2_dgemm("N", "N", 4, 4, 4, 1.0, A, 4, A, 4, 0.0, C, 4, variant=99, check=False) == 1004
+    torch.cuda.synchronize()
+    assert (C == 1).all()
+
+
+@pytest.mark.parametrize("kind", ["d", "s"])
+def test_deterministic_bitwise(b2, kind):
+    """Two runs of the same problem give the same bits (no races in the accumulation)."""
+    tdt = torch.float64 if kind == "d" else torch.float32
+    fn = b2.b2_dgemm if kind == "d" else b2.b2_sgemm
+    m, n, k = 777, 513, 1031
+    A, lda, B, ldb, C, ldc = synth.gemm_inputs("T", "N", m, n, k, "uniform", 77, tdt)
+    outs = []
+    for _ in range(2):
+        Cd = C.cuda()
+        fn("T", "N", m, n, k, 0.7, A.cuda(), lda, B.cuda(), ldb, -0.3, Cd, ldc)
+        outs.append(Cd.cpu())
+    assert torch.equal(outs[0].view(torch.uint8), outs[1].view(torch.uint8))
+
+
+# ---- complex 4M ------------------------------------------------------------------------------------
+
+def test_zgemm4m_small_full_all_transposes(b2, oracle):
+    for ta, tb in TRANS:
+        run_and_check(b2, oracle, "z", ta, tb, 301, 203, 157, 1 + 0.5j, 0j, seed=51, pad=True)
+        run_and_check(b2, oracle, "z", ta, tb, 130, 70, 33, 0.3 - 0.8j, 0.25 + 0.75j, seed=52, pad=True)
+        run_and_check(b2, oracle, "z", ta, tb, 130, 70, 33, 2 - 1j, 0.5 + 0.5j, dist="int9", seed=53,
+                      expect_exact=True)
+    run_and_check(b2, oracle, "z", "N", "N", 33, 17, 0, 1 + 1j, 0.5 - 0.5j, seed=54)
+    run_and_check(b2, oracle, "z", "N", "N", 33, 17, 9, 0j, 0.5 - 0.5j, seed=55)
+    run_and_check(b2, oracle, "z", "N", "N", 0, 17, 9, 1 + 0j, 0j, seed=56)
+
+
+def test_zgemm4m_argument_errors(b2):
+    z = torch.zeros(64, dtype=torch.complex128, device="cuda")
+    ws = torch.empty(1 << 16, dtype=torch.uint8, device="cuda")
+    assert b2.b2_zgemm4m("C", "N", 4, 4, 4, 1, z, 4, z, 4, 0, z, 4, ws, check=False) == -1
+    assert b2.b2_zgemm4m("N", "C", 4, 4, 4, 1, z, 4, z, 4, 0, z, 4, ws, check=False) == -2
+    assert b2.b2_zgemm4m("N", "N", 4, 4, 4, 1, z, 4, z, 4, 0, z, 4, None, check=False) == 1003
+    assert b2.b2_zgemm4m("N", "N", 4, 4, 4, 1, z, 4, z, 4, 0, z, 4, ws[:64], check=False) == 1003
+    assert b2.b2_zgemm4m("N", "N", 4, 4, 4, 1, z, 4, z, 4, 0, z, 4, ws[8:], check=False) == 1003  # misaligned
+
+
+# ---- host-buffer entry points ----------------------------------------------------------------------
+
+@pytest.mark.parametrize("kind", ["d", "s"])
+def test_host_entry_matches_oracle(b2, oracle, kind):
+    tdt = torch.float64 if kind == "d" else torch.float32
+    fn = b2.b2_dgemm_host if kind == "d" else b2.b2_sgemm_host
+    u = 2.0 ** -53 if kind == "d" else 2.0 ** -24
+    for ta, tb in TRANS:
+        m, n, k = 301, 203, 157
+        (ra, ca), (rb, cb) = synth.operand_shapes(ta, tb, m, n, k)
+        A, lda, B, ldb, C, ldc = synth.gemm_inputs(ta, tb, m, n, k, "uniform", 61, tdt, ra + 5, rb + 3, m + 7)
+        want = C.numpy().copy()
+        oracle.ref_gemm(ta, tb, m, n, k, 0.7, A.numpy(), lda, B.numpy(), ldb, -0.3, want, ldc)
+        _, S = oracle.ref_gemm_hi(ta, tb, m, n, k, 0.7, A.numpy(), lda, B.numpy(), ldb, -0.3, C.numpy(), ldc)
+        ws = torch.empty(b2.b2_gemm_host_workspace_bytes(0 if kind == "d" else 1, ta, tb, m, n, k), dtype=torch.uint8,
+                         device="cuda")
+        Ch = C.clone().pin_memory()
+        fn(ta, tb, m, n, k, 0.7, A.pin_memory(), lda, B.pin_memory(), ldb, -0.3, Ch, ldc, ws)
+        got = Ch.numpy().reshape(n, ldc)
+        assert got[:, m:].tobytes() == C.numpy().reshape(n, ldc)[:, m:].tobytes()
+        err = np.abs(got[:, :m].astype(np.float64) - want.reshape(n, ldc)[:, :m].astype(np.float64))
+        assert np.all(err <= 2 * k * u * S.reshape(n, m))
+
+
+# ---- selector and probe ----------------------------------------------------------------------------
+
+def test_query_config_reports_launch(b2):
+    import json
+    cfg = json.loads(b2.b2_gemm_query_config(0, "N", "N", 8192, 8192, 8192, 8192, 8192, 8192))
+    assert cfg["micro_kernel"] == "dmma" and cfg["grid"] == cfg["tiles_m"] * cfg["tiles_n"]
+    assert cfg["tiles_m"] == -(-8192 // cfg["BM"]) and cfg["k_slabs"] == 8192 // cfg["kc"]
+    cfg = json.loads(b2.b2_gemm_query_config(1, "T", "N", 1001, 999, 1003, 1027, 1027, 1027))
+    assert cfg["micro_kernel"] == "ffma" and cfg["vector_staging_if_pointers_aligned"] is False
+
+
+def test_pipe_probe_rates(b2):
+    from paper_1611_08035_b200 import pipes
+    d = pipes.probe("dfma", 256, 1, 4000)
+    t = pipes.probe("dmma_m16n8k4", 256, 1, 2000)
+    f = pipes.probe("ffma", 256, 1, 4000)
+    assert 55 <= d["fma_per_clk_per_sm"] <= 66 and 55 <= t["fma_per_clk_per_sm"] <= 66
+    assert 110 <= f["fma_per_clk_per_sm"] <= 132
