@@ -1,5 +1,6 @@
 // C-ABI entry points of the real GEMM: argument checking, quick returns, variant selection.
 #include <cuda_runtime.h>
+#include <math.h>
 #include <stdio.h>
 #include <string.h>
 
@@ -140,7 +141,12 @@ int gemm_entry(int variant, char transa, char transb, int64_t m, int64_t n, int6
   args.alpha = alpha, args.beta = beta;
   args.A = A, args.lda = lda, args.B = B, args.ldb = ldb, args.C = C, args.ldc = ldc;
   args.tiles_m = args.tiles_n = 0;
-  args.group_m = 8;
+  // Rasterisation group: the CTAs resident at one time should cover a block of C whose A row-panels and
+  // B column-panels have about the same size: group_m * BM = (resident / group_m) * BN.
+  const VariantInfo& vi = variant_info_t<T>(variant);
+  const double resident = (double)sm_count_cached() * vi.ctas_per_sm;
+  int group_m = (int)(sqrt(resident * vi.bn / vi.bm) + 0.5);
+  args.group_m = group_m < 1 ? 1 : group_m;
   return variant_launch_t<T>(variant)(args, is_t(transa), is_t(transb), operands_aligned(A, lda, B, ldb), stream);
 }
 

@@ -29,61 +29,97 @@ enum Layout { OC = 0, KC = 1 };
 
 // ---------------------------------------------------------------------------------------
 // Staging of one BO x BK operand tile from global memory into shared memory with cp.async.
-// X0 points at element (o0, k0) of the operand; o_valid / k_valid are the numbers of valid
-// rows and k-entries from there (anything beyond is zero-filled and never read from global).
+//
+// Two paths.  The fast path serves slabs that lie completely inside the operand (the steady
+// state of interior tiles): every thread keeps one running source pointer, the chunk
+// addresses differ from it by compile-time multiples of one hoisted stride, and nothing is
+// predicated.  The general path serves edge tiles and the last, partial k-slab: every chunk
+// is clipped against the valid extents, zero-filled beyond them and never read from global.
 // VEC is the number of elements per cp.async when source and destination layouts agree
-// (16-byte chunks need 16-byte aligned columns); element-wise copies transpose on the fly.
+// (16-byte chunks need 16-byte aligned columns); when they differ (k-contiguous source packed
+// into the OC layout) the copy is element-wise and transposes on the fly.
 // ---------------------------------------------------------------------------------------
 template <typename T, int BO, int BK, int NT, Layout SRC, Layout DST, int VEC, int PITCH>
 struct Stager {
   static constexpr int ELEM = sizeof(T);
+  static constexpr bool STRAIGHT = (SRC == DST);
+  static_assert(STRAIGHT || (SRC == KC && DST == OC), "only k-contiguous sources are transposed while staging");
+  static constexpr int RUN = 8;  // transposing copy: run length along k handled by consecutive threads
+  // straight copy geometry
+  static constexpr int CE = (SRC == OC) ? BO : BK;  // contiguous extent
+  static constexpr int OE = (SRC == OC) ? BK : BO;  // number of lines
+  static constexpr int CPL = CE / VEC;              // chunks per line
+  static constexpr int TOTAL = STRAIGHT ? OE * CPL : BO * BK;
+  static constexpr int ITER = (TOTAL + NT - 1) / NT;
+  static_assert(!STRAIGHT || CE % VEC == 0, "tile extent must be a multiple of the chunk");
+  static_assert(TOTAL % NT == 0, "every thread copies the same number of chunks");
+  static_assert(!STRAIGHT || NT % CPL == 0, "a line must be covered by consecutive threads of one pass");
+  static constexpr int LSTEP = STRAIGHT ? NT / CPL : NT / RUN;  // lines (straight) or o-rows (transposing) per pass
+  static constexpr int Q = STRAIGHT ? 1 : BO / LSTEP;           // transposing: passes that cover the o-extent once
+  static_assert(STRAIGHT || (NT % RUN == 0 && BO % LSTEP == 0 && BK % RUN == 0), "transposing copy geometry");
 
-  static __device__ __forceinline__ void load(T* __restrict__ s, const T* __restrict__ X0, int64_t ld, int o_valid,
-                                              int k_valid, int tid) {
-    if constexpr (SRC == DST) {
-      constexpr int CE = (SRC == OC) ? BO : BK;  // contiguous extent
-      constexpr int OE = (SRC == OC) ? BK : BO;  // number of lines
-      constexpr int CPL = CE / VEC;              // chunks per line
-      constexpr int TOTAL = OE * CPL;
-      constexpr int ITER = (TOTAL + NT - 1) / NT;
-      static_assert(CE % VEC == 0, "tile extent must be a multiple of the chunk");
+  const T* src;    // this thread's first chunk of the next slab to stage
+  int64_t lstep;   // source elements between the lines of consecutive passes
+  int64_t kstep;   // source elements to advance by one slab (BK along k)
+  int dst0;        // element offset of this thread's first chunk inside a stage
+
+  __device__ __forceinline__ void init(const T* X0, int64_t ld, int tid) {
+    lstep = (int64_t)LSTEP * ld;
+    if constexpr (STRAIGHT) {
+      const int line = tid / CPL, cc = (tid % CPL) * VEC;
+      src = X0 + cc + (int64_t)line * ld;
+      dst0 = line * PITCH + cc;
+      kstep = (SRC == OC) ? (int64_t)BK * ld : (int64_t)BK;
+    } else {
+      const int kk = tid % RUN, o = tid / RUN;
+      src = X0 + kk + (int64_t)o * ld;
+      dst0 = kk * PITCH + o;
+      kstep = BK;
+    }
+  }
+
+  __device__ __forceinline__ void advance() { src += kstep; }
+
+  // Slab fully inside the operand: no predicates.
+  __device__ __forceinline__ void load_fast(T* __restrict__ s) const {
+#pragma unroll
+    for (int it = 0; it < ITER; ++it) {
+      if constexpr (STRAIGHT) {
+        cp_async_zfill<VEC * ELEM>(s + dst0 + it * LSTEP * PITCH, src + it * lstep, VEC * ELEM);
+      } else {
+        const int a = it % Q, b = it / Q;
+        cp_async_zfill<ELEM>(s + dst0 + b * RUN * PITCH + a * LSTEP, src + a * lstep + b * RUN, ELEM);
+      }
+    }
+  }
+
+  // General path.  X0 points at element (o0, k0) of the operand; o_valid / k_valid are the numbers of valid
+  // rows and k-entries from there.
+  static __device__ __noinline__ void load_general(T* __restrict__ s, const T* __restrict__ X0, int64_t ld,
+                                                   int o_valid, int k_valid, int tid) {
+    if constexpr (STRAIGHT) {
       const int c_valid = (SRC == OC) ? o_valid : k_valid;
       const int l_valid = (SRC == OC) ? k_valid : o_valid;
-#pragma unroll
+#pragma unroll 1
       for (int it = 0; it < ITER; ++it) {
         const int c = tid + it * NT;
-        if (TOTAL % NT != 0 && c >= TOTAL) break;
         const int line = c / CPL;
         const int cc = (c % CPL) * VEC;
         int nvalid = c_valid - cc;
         nvalid = nvalid < 0 ? 0 : (nvalid > VEC ? VEC : nvalid);
         if (line >= l_valid) nvalid = 0;
-        const T* src = nvalid > 0 ? X0 + cc + (int64_t)line * ld : X0;
-        cp_async_zfill<VEC * ELEM>(s + line * PITCH + cc, src, nvalid * ELEM);
+        const T* g = nvalid > 0 ? X0 + cc + (int64_t)line * ld : X0;
+        cp_async_zfill<VEC * ELEM>(s + line * PITCH + cc, g, nvalid * ELEM);
       }
     } else {
-      // element-wise transposing copy; runs of 8 along the source's contiguous dimension
-      constexpr int TOTAL = BO * BK;
-      constexpr int ITER = (TOTAL + NT - 1) / NT;
-      constexpr int RUN = 8;
-      static_assert(BK % RUN == 0 && BO % RUN == 0, "tile extents must be multiples of 8");
-#pragma unroll
+#pragma unroll 1
       for (int it = 0; it < ITER; ++it) {
         const int c = tid + it * NT;
-        if (TOTAL % NT != 0 && c >= TOTAL) break;
-        int o, kk;
-        if constexpr (SRC == KC) {  // source k-contiguous
-          kk = (c % RUN) + RUN * (c / (RUN * BO));
-          o = (c / RUN) % BO;
-        } else {  // source o-contiguous
-          o = (c % RUN) + RUN * (c / (RUN * BK));
-          kk = (c / RUN) % BK;
-        }
+        const int kk = (c % RUN) + RUN * (c / (RUN * BO));
+        const int o = (c / RUN) % BO;
         const bool ok = (o < o_valid) && (kk < k_valid);
-        const T* src = X0;
-        if (ok) src = (SRC == KC) ? X0 + kk + (int64_t)o * ld : X0 + o + (int64_t)kk * ld;
-        T* dst = (DST == OC) ? s + kk * PITCH + o : s + o * PITCH + kk;
-        cp_async_zfill<ELEM>(dst, src, ok ? ELEM : 0);
+        const T* g = ok ? X0 + kk + (int64_t)o * ld : X0;
+        cp_async_zfill<ELEM>(s + kk * PITCH + o, g, ok ? ELEM : 0);
       }
     }
   }
@@ -362,18 +398,37 @@ struct GemmKernel {
     const int64_t stepB = TB ? (int64_t)BK * p.ldb : (int64_t)BK;
 
     const int KT = (int)((p.k + BK - 1) / BK);
+    const int k_tail = (int)(p.k - (int64_t)(KT - 1) * BK);  // valid k-entries of the last slab
+    const bool a_inside = (m_valid == BM), b_inside = (n_valid == BN);
 
-    auto stage = [&](int kt) {
-      const int slot = kt % STAGES;
-      const int k_valid = (int)min((int64_t)BK, p.k - (int64_t)kt * BK);
-      StageA::load(sA + slot * Micro::A_STAGE, gA + kt * stepA, p.lda, m_valid, k_valid, tid);
-      StageB::load(sB + slot * Micro::B_STAGE, gB + kt * stepB, p.ldb, n_valid, k_valid, tid);
+    StageA stA;
+    StageB stB;
+    stA.init(gA, p.lda, tid);
+    stB.init(gB, p.ldb, tid);
+
+    // stage slab kt (slabs are staged in increasing order, so the running pointers follow along)
+    auto stage = [&](int kt, int slot) {
+      const int k_valid = (kt == KT - 1) ? k_tail : BK;
+      T* dA = sA + slot * Micro::A_STAGE;
+      T* dB = sB + slot * Micro::B_STAGE;
+      if (a_inside && k_valid == BK) {
+        stA.load_fast(dA);
+      } else {
+        StageA::load_general(dA, gA + kt * stepA, p.lda, m_valid, k_valid, tid);
+      }
+      if (b_inside && k_valid == BK) {
+        stB.load_fast(dB);
+      } else {
+        StageB::load_general(dB, gB + kt * stepB, p.ldb, n_valid, k_valid, tid);
+      }
+      stA.advance();
+      stB.advance();
     };
 
     // ramp-up: fill STAGES-1 slots (the first of the paper's three stages of the k-loop)
 #pragma unroll
     for (int s = 0; s < STAGES - 1; ++s) {
-      if (s < KT) stage(s);
+      if (s < KT) stage(s, s);
       cp_async_commit();
     }
 
@@ -381,14 +436,15 @@ struct GemmKernel {
     Micro::zero(acc);
 
     // steady state: wait for slab kt, refill the slot freed in the previous iteration, compute
+    int slot = 0, fill = STAGES - 1;
     for (int kt = 0; kt < KT; ++kt) {
       cp_async_wait<STAGES - 2>();
       __syncthreads();
-      const int next = kt + STAGES - 1;
-      if (next < KT) stage(next);
+      if (kt + STAGES - 1 < KT) stage(kt + STAGES - 1, fill);
       cp_async_commit();
-      const int slot = kt % STAGES;
       Micro::compute(acc, sA + slot * Micro::A_STAGE, sB + slot * Micro::B_STAGE, warp_m, warp_n, lane);
+      slot = (slot + 1 == STAGES) ? 0 : slot + 1;
+      fill = (fill + 1 == STAGES) ? 0 : fill + 1;
     }
     cp_async_wait<0>();
 
