@@ -212,41 +212,64 @@ struct DmmaMicro {
   }
 
   // C := alpha*acc + beta*C on the warp's block; rows >= m and columns >= n are skipped.
+  // The old C values are fetched in batches, all loads of a batch issued before the first
+  // store, so their latencies overlap instead of adding up (a store to C may alias a later
+  // load of C as far as the compiler can tell).
   static __device__ __forceinline__ void epilogue(const Acc& acc, const GemmArgs<double>& p, int64_t m0, int64_t n0,
                                                   int warp_m, int warp_n, int lane) {
     const int g = lane >> 2, t = lane & 3;
     const bool vec_ok = ((reinterpret_cast<uintptr_t>(p.C) & 15) == 0) && ((p.ldc & 1) == 0);
     const bool use_beta = (p.beta != 0.0);
+    // old values in flight per batch: 32 doubles when the register budget is 255, 16 when it is 128
+    constexpr int BATCH = (MI * NI * 4 >= 64) ? 32 : 16;
+    constexpr int NB = (BATCH / (MI * 4)) > 0 ? ((BATCH / (MI * 4)) < NI ? (BATCH / (MI * 4)) : NI) : 1;
+    static_assert(NI % NB == 0, "batches must tile the fragment columns");
+    const int64_t row0 = m0 + warp_m * WTM + 2 * g;
+    const int64_t col0 = n0 + warp_n * WTN + 2 * t;
 #pragma unroll
-    for (int ni = 0; ni < NI; ++ni) {
+    for (int nb0 = 0; nb0 < NI; nb0 += NB) {
+      double2 old[NB][2][MI];
+      if (use_beta) {
 #pragma unroll
-      for (int h = 0; h < 2; ++h) {
-        const int64_t col = n0 + warp_n * WTN + ni * 8 + 2 * t + h;
-        if (col >= p.n) continue;
-        double* ccol = p.C + col * p.ldc;
+        for (int nb = 0; nb < NB; ++nb)
 #pragma unroll
-        for (int mi = 0; mi < MI; ++mi) {
-          const int64_t row = m0 + warp_m * WTM + mi * 16 + 2 * g;
-          if (row >= p.m) continue;
-          double v0 = p.alpha * acc.c[mi][ni][h], v1 = p.alpha * acc.c[mi][ni][2 + h];
-          double* dst = ccol + row;
-          if (vec_ok && row + 1 < p.m) {
-            if (use_beta) {
-              const double2 old = *reinterpret_cast<const double2*>(dst);
-              v0 += p.beta * old.x;
-              v1 += p.beta * old.y;
+          for (int h = 0; h < 2; ++h)
+#pragma unroll
+            for (int mi = 0; mi < MI; ++mi) {
+              const int64_t col = col0 + (nb0 + nb) * 8 + h, row = row0 + mi * 16;
+              old[nb][h][mi] = make_double2(0.0, 0.0);
+              if (col < p.n && row < p.m) {
+                const double* src = p.C + col * p.ldc + row;
+                if (vec_ok && row + 1 < p.m) {
+                  old[nb][h][mi] = *reinterpret_cast<const double2*>(src);
+                } else {
+                  old[nb][h][mi].x = src[0];
+                  if (row + 1 < p.m) old[nb][h][mi].y = src[1];
+                }
+              }
             }
-            *reinterpret_cast<double2*>(dst) = make_double2(v0, v1);
-          } else {
-            if (use_beta) v0 += p.beta * dst[0];
-            dst[0] = v0;
-            if (row + 1 < p.m) {
-              if (use_beta) v1 += p.beta * dst[1];
-              dst[1] = v1;
+      }
+#pragma unroll
+      for (int nb = 0; nb < NB; ++nb)
+#pragma unroll
+        for (int h = 0; h < 2; ++h)
+#pragma unroll
+          for (int mi = 0; mi < MI; ++mi) {
+            const int64_t col = col0 + (nb0 + nb) * 8 + h, row = row0 + mi * 16;
+            if (col >= p.n || row >= p.m) continue;
+            double v0 = p.alpha * acc.c[mi][nb0 + nb][h], v1 = p.alpha * acc.c[mi][nb0 + nb][2 + h];
+            if (use_beta) {
+              v0 += p.beta * old[nb][h][mi].x;
+              v1 += p.beta * old[nb][h][mi].y;
+            }
+            double* dst = p.C + col * p.ldc + row;
+            if (vec_ok && row + 1 < p.m) {
+              *reinterpret_cast<double2*>(dst) = make_double2(v0, v1);
+            } else {
+              dst[0] = v0;
+              if (row + 1 < p.m) dst[1] = v1;
             }
           }
-        }
-      }
     }
   }
 };
@@ -314,45 +337,69 @@ struct SimtMicro {
     }
   }
 
+  // C := alpha*acc + beta*C; old C values are fetched in batches of columns before any store of the batch.
   static __device__ __forceinline__ void epilogue(const Acc& acc, const GemmArgs<T>& p, int64_t m0, int64_t n0,
                                                   int warp_m, int warp_n, int lane) {
     const int lx = lane & 7, ly = lane >> 3;
     const bool vec_ok = ((reinterpret_cast<uintptr_t>(p.C) & 15) == 0) && ((p.ldc % VEC) == 0);
     const bool use_beta = (p.beta != T(0));
+    constexpr int JB = 2;  // columns per batch: 16 old values in flight
+    const int64_t row0 = m0 + warp_m * WTM + lx * VEC;
+    const int64_t col0 = n0 + warp_n * WTN + ly * VEC;
 #pragma unroll
-    for (int j = 0; j < TN; ++j) {
-      const int64_t col = n0 + warp_n * WTN + (j / VEC) * 4 * VEC + ly * VEC + (j % VEC);
-      if (col >= p.n) continue;
-      T* ccol = p.C + col * p.ldc;
+    for (int j0 = 0; j0 < TN; j0 += JB) {
+      T old[JB][TM];
+      if (use_beta) {
 #pragma unroll
-      for (int gi = 0; gi < TM / VEC; ++gi) {
-        const int64_t row = m0 + warp_m * WTM + gi * 8 * VEC + lx * VEC;
-        if (row >= p.m) continue;
-        T v[VEC];
+        for (int jb = 0; jb < JB; ++jb) {
+          const int j = j0 + jb;
+          const int64_t col = col0 + (j / VEC) * 4 * VEC + (j % VEC);
 #pragma unroll
-        for (int e = 0; e < VEC; ++e) v[e] = p.alpha * acc.c[gi * VEC + e][j];
-        T* dst = ccol + row;
-        if (vec_ok && row + VEC <= p.m) {
-          if (use_beta) {
-            T old[VEC];
-            load_vec(old, dst);
+          for (int gi = 0; gi < TM / VEC; ++gi) {
+            const int64_t row = row0 + gi * 8 * VEC;
 #pragma unroll
-            for (int e = 0; e < VEC; ++e) v[e] += p.beta * old[e];
+            for (int e = 0; e < VEC; ++e) old[jb][gi * VEC + e] = T(0);
+            if (col < p.n && row < p.m) {
+              const T* src = p.C + col * p.ldc + row;
+              if (vec_ok && row + VEC <= p.m) {
+                load_vec(&old[jb][gi * VEC], src);
+              } else {
+#pragma unroll
+                for (int e = 0; e < VEC; ++e)
+                  if (row + e < p.m) old[jb][gi * VEC + e] = src[e];
+              }
+            }
           }
-          VT out;
-          if constexpr (sizeof(T) == 4) {
-            out = make_float4(v[0], v[1], v[2], v[3]);
-          } else {
-            out = make_double2(v[0], v[1]);
-          }
-          *reinterpret_cast<VT*>(dst) = out;
-        } else {
+        }
+      }
+#pragma unroll
+      for (int jb = 0; jb < JB; ++jb) {
+        const int j = j0 + jb;
+        const int64_t col = col0 + (j / VEC) * 4 * VEC + (j % VEC);
+        if (col >= p.n) continue;
+#pragma unroll
+        for (int gi = 0; gi < TM / VEC; ++gi) {
+          const int64_t row = row0 + gi * 8 * VEC;
+          if (row >= p.m) continue;
+          T v[VEC];
 #pragma unroll
           for (int e = 0; e < VEC; ++e) {
-            if (row + e < p.m) {
-              if (use_beta) v[e] += p.beta * dst[e];
-              dst[e] = v[e];
+            v[e] = p.alpha * acc.c[gi * VEC + e][j];
+            if (use_beta) v[e] += p.beta * old[jb][gi * VEC + e];
+          }
+          T* dst = p.C + col * p.ldc + row;
+          if (vec_ok && row + VEC <= p.m) {
+            VT out;
+            if constexpr (sizeof(T) == 4) {
+              out = make_float4(v[0], v[1], v[2], v[3]);
+            } else {
+              out = make_double2(v[0], v[1]);
             }
+            *reinterpret_cast<VT*>(dst) = out;
+          } else {
+#pragma unroll
+            for (int e = 0; e < VEC; ++e)
+              if (row + e < p.m) dst[e] = v[e];
           }
         }
       }
