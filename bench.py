@@ -293,7 +293,8 @@ def main():
     w = WORKLOAD
     m, n, k = w["m"], w["n"], w["k"]
     flops = 2.0 * m * n * k
-    A, lda, B, ldb, C, ldc = device_inputs(w, torch.float64, device, seed_shift=1000 * rank)
+    from paper_1611_08035_b200 import replicas
+    A, lda, B, ldb, C, ldc = device_inputs(w, torch.float64, device, seed_shift=replicas.rank_seed(0, rank))
 
     def step():
         b2.b2_dgemm(w["transa"], w["transb"], m, n, k, w["alpha"], A, lda, B, ldb, w["beta"], C, ldc)
@@ -304,11 +305,7 @@ def main():
         time.sleep(0.3)
     total_ms, per_step = time_steps(step, args.steps, args.warmup, barrier)
     clocks = sampler.stop() if rank == 0 else None
-    if world > 1:
-        t = torch.tensor([total_ms], device=device, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
-    value = world * flops * args.steps / (total_ms * 1e-3) / 1e9
+    value, total_ms = replicas.aggregate_gflops(flops, args.steps, total_ms, world, dist, device)
     kernel_ms = statistics.mean(per_step)
 
     # end to end: host buffers in, result back in host memory, through the host-buffer C entry point
@@ -326,11 +323,7 @@ def main():
     for _ in range(e2e_steps):
         e2e_step()  # synchronises the stream before returning
     e2e_s = time.perf_counter() - t0
-    if world > 1:
-        t = torch.tensor([e2e_s], device=device, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
-    e2e_value = world * flops * e2e_steps / e2e_s / 1e9
+    e2e_value, _ = replicas.aggregate_gflops(flops, e2e_steps, e2e_s * 1e3, world, dist, device)
     elem = 8
     h2d = (m * k + k * n + m * n) * elem
     d2h = m * n * elem
