@@ -144,6 +144,7 @@ int b2_sgemm_host(char transa, char transb, int64_t m, int64_t n, int64_t k, flo
 #define B2_PROBE_DMMA_M16N8K4 3
 #define B2_PROBE_DMMA_M16N8K8 4
 #define B2_PROBE_DMMA_M16N8K16 5
+#define B2_PROBE_FFMA2 6 /* packed fp32 pair multiply-add, fma.rn.f32x2 */
 int b2_pipe_probe(int kind, int threads_per_cta, int ctas, int64_t iters, void* scratch, size_t scratch_bytes,
                   double* fma_per_thread_iter, void* cuda_stream);
 

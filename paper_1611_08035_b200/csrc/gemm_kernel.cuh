@@ -298,15 +298,38 @@ struct SimtMicro {
   static constexpr int A_STAGE = BK * PA, B_STAGE = BK * PB;
   using VT = typename std::conditional<sizeof(T) == 4, float4, double2>::type;
 
-  struct Acc {
+  // Accumulators: scalar c[i][j] for fp64; for fp32 packed row pairs p[i/2][j] = (c[i][j], c[i+1][j]), i even.
+  struct AccScalar {
     T c[TM][TN];
   };
+  struct AccPairs {
+    unsigned long long p[TM / 2][TN];
+  };
+  using Acc = typename std::conditional<sizeof(T) == 4, AccPairs, AccScalar>::type;
 
   static __device__ __forceinline__ void zero(Acc& acc) {
+    if constexpr (sizeof(T) == 4) {
 #pragma unroll
-    for (int i = 0; i < TM; ++i)
+      for (int i = 0; i < TM / 2; ++i)
 #pragma unroll
-      for (int j = 0; j < TN; ++j) acc.c[i][j] = T(0);
+        for (int j = 0; j < TN; ++j) acc.p[i][j] = 0ull;
+    } else {
+#pragma unroll
+      for (int i = 0; i < TM; ++i)
+#pragma unroll
+        for (int j = 0; j < TN; ++j) acc.c[i][j] = T(0);
+    }
+  }
+
+  // accumulator element (i, j)
+  static __device__ __forceinline__ T get(const Acc& acc, int i, int j) {
+    if constexpr (sizeof(T) == 4) {
+      float lo, hi;
+      asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(acc.p[i / 2][j]));
+      return (i & 1) ? hi : lo;
+    } else {
+      return acc.c[i][j];
+    }
   }
 
   static __device__ __forceinline__ void load_vec(T* dst, const T* src) {
@@ -323,17 +346,46 @@ struct SimtMicro {
     const int lx = lane & 7, ly = lane >> 3;
     const T* pa = sA + warp_m * WTM + lx * VEC;
     const T* pb = sB + warp_n * WTN + ly * VEC;
+    if constexpr (sizeof(T) == 4) {
+      // FP32: packed pair multiply-adds (fma.rn.f32x2, two IEEE fp32 FMAs per instruction).  A pair holds two
+      // adjacent rows of one column of the accumulator block; a is used pairwise as loaded, b is duplicated
+      // into both halves.  32 instructions instead of 64 per outer product: the FP32 pipe stays busy while
+      // half of the issue slots are free for the shared-memory loads and the staging code.
 #pragma unroll
-    for (int kk = 0; kk < BK; ++kk) {
-      T a[TM], b[TN];
+      for (int kk = 0; kk < BK; ++kk) {
+        unsigned long long ap[TM / 2], bd[TN];
 #pragma unroll
-      for (int gi = 0; gi < TM / VEC; ++gi) load_vec(a + gi * VEC, pa + kk * PA + gi * 8 * VEC);
+        for (int gi = 0; gi < TM / VEC; ++gi) {
+          const ulonglong2 v = *reinterpret_cast<const ulonglong2*>(pa + kk * PA + gi * 8 * VEC);
+          ap[2 * gi] = v.x, ap[2 * gi + 1] = v.y;
+        }
 #pragma unroll
-      for (int gj = 0; gj < TN / VEC; ++gj) load_vec(b + gj * VEC, pb + kk * PB + gj * 4 * VEC);
+        for (int gj = 0; gj < TN / VEC; ++gj) {
+          const float4 v = *reinterpret_cast<const float4*>(pb + kk * PB + gj * 4 * VEC);
+          asm("mov.b64 %0, {%1, %1};" : "=l"(bd[4 * gj + 0]) : "f"(v.x));
+          asm("mov.b64 %0, {%1, %1};" : "=l"(bd[4 * gj + 1]) : "f"(v.y));
+          asm("mov.b64 %0, {%1, %1};" : "=l"(bd[4 * gj + 2]) : "f"(v.z));
+          asm("mov.b64 %0, {%1, %1};" : "=l"(bd[4 * gj + 3]) : "f"(v.w));
+        }
 #pragma unroll
-      for (int i = 0; i < TM; ++i)
+        for (int ip = 0; ip < TM / 2; ++ip)
 #pragma unroll
-        for (int j = 0; j < TN; ++j) acc.c[i][j] = fma(a[i], b[j], acc.c[i][j]);
+          for (int j = 0; j < TN; ++j)
+            asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(acc.p[ip][j]) : "l"(ap[ip]), "l"(bd[j]));
+      }
+    } else {
+#pragma unroll
+      for (int kk = 0; kk < BK; ++kk) {
+        T a[TM], b[TN];
+#pragma unroll
+        for (int gi = 0; gi < TM / VEC; ++gi) load_vec(a + gi * VEC, pa + kk * PA + gi * 8 * VEC);
+#pragma unroll
+        for (int gj = 0; gj < TN / VEC; ++gj) load_vec(b + gj * VEC, pb + kk * PB + gj * 4 * VEC);
+#pragma unroll
+        for (int i = 0; i < TM; ++i)
+#pragma unroll
+          for (int j = 0; j < TN; ++j) acc.c[i][j] = fma(a[i], b[j], acc.c[i][j]);
+      }
     }
   }
 
@@ -384,7 +436,7 @@ struct SimtMicro {
           T v[VEC];
 #pragma unroll
           for (int e = 0; e < VEC; ++e) {
-            v[e] = p.alpha * acc.c[gi * VEC + e][j];
+            v[e] = p.alpha * get(acc, gi * VEC + e, j);
             if (use_beta) v[e] += p.beta * old[jb][gi * VEC + e];
           }
           T* dst = p.C + col * p.ldc + row;
@@ -452,6 +504,20 @@ struct GemmKernel {
     StageB stB;
     stA.init(gA, p.lda, tid);
     stB.init(gB, p.ldb, tid);
+
+    // beta != 0: pull this tile's old C values towards L2 now, so that the epilogue's loads overlap the k-loop
+    // instead of paying the DRAM latency after it (this matters when k is only a few slabs).
+    if (p.beta != T(0)) {
+      constexpr int LINE = 128 / (int)sizeof(T);   // elements per 128-byte line
+      constexpr int LPC = (BM + LINE - 1) / LINE;  // lines per tile column
+      for (int c = tid; c < BN * LPC; c += NT) {
+        const int col = c / LPC, row = (c % LPC) * LINE;
+        if (col < n_valid && row < m_valid) {
+          const T* ptr = p.C + (n0 + col) * p.ldc + m0 + row;
+          asm volatile("prefetch.global.L2 [%0];" ::"l"(ptr));
+        }
+      }
+    }
 
     // stage slab kt (slabs are staged in increasing order, so the running pointers follow along)
     auto stage = [&](int kt, int slot) {

@@ -11,6 +11,7 @@ struct VariantInfo {
   const char* name;
   const char* micro;  // "dmma" | "dfma" | "ffma"
   int bm, bn, bk, stages, threads, ctas_per_sm;
+  double efficiency;  // measured steady-state fraction of the arithmetic pipe's peak (large interior problems)
 };
 
 template <typename T>

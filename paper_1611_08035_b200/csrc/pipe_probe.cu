@@ -52,6 +52,35 @@ __global__ void probe_ffma(long long iters, float* sink, long long* cycles) {
   if (threadIdx.x == 0) cycles[blockIdx.x] = t1 - t0;
 }
 
+// Packed FP32 pair FMA (fma.rn.f32x2, sm_100+): two IEEE fp32 multiply-adds per thread per instruction.
+__global__ void probe_ffma2(long long iters, float* sink, long long* cycles) {
+  unsigned long long acc[kAcc / 2];
+  unsigned long long a, b;
+  const float af = 1.0f + 1e-6f * threadIdx.x, bf = 1e-9f;
+  asm volatile("mov.b64 %0, {%1, %1};" : "=l"(a) : "f"(af));
+  asm volatile("mov.b64 %0, {%1, %1};" : "=l"(b) : "f"(bf));
+#pragma unroll
+  for (int i = 0; i < kAcc / 2; ++i) {
+    const float v = 1.0f + i;
+    asm volatile("mov.b64 %0, {%1, %1};" : "=l"(acc[i]) : "f"(v));
+  }
+  long long t0 = clock64();
+  for (long long it = 0; it < iters; ++it) {
+#pragma unroll
+    for (int i = 0; i < kAcc / 2; ++i) asm volatile("fma.rn.f32x2 %0, %0, %1, %2;" : "+l"(acc[i]) : "l"(a), "l"(b));
+  }
+  long long t1 = clock64();
+  float s = 0;
+#pragma unroll
+  for (int i = 0; i < kAcc / 2; ++i) {
+    float lo, hi;
+    asm volatile("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(acc[i]));
+    s += lo + hi;
+  }
+  if (s == 123.456f) sink[0] = s;
+  if (threadIdx.x == 0) cycles[blockIdx.x] = t1 - t0;
+}
+
 // DMMA probes: NSETS independent accumulator fragments per warp, A/B fragments fixed.
 template <int NSETS>
 __global__ void probe_dmma_m8n8k4(long long iters, double* sink, long long* cycles) {
@@ -168,6 +197,10 @@ extern "C" int b2_pipe_probe(int kind, int threads_per_cta, int ctas, int64_t it
       break;
     case B2_PROBE_FFMA:
       probe_ffma<<<ctas, threads_per_cta, 0, st>>>(iters, (float*)sink, cyc);
+      *fma_per_thread_iter = kAcc;
+      break;
+    case B2_PROBE_FFMA2:
+      probe_ffma2<<<ctas, threads_per_cta, 0, st>>>(iters, (float*)sink, cyc);
       *fma_per_thread_iter = kAcc;
       break;
     case B2_PROBE_DMMA_M8N8K4:

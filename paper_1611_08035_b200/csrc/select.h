@@ -15,6 +15,7 @@ struct TileChoice {
   int bm, bn, bk;
   int threads;
   int ctas_per_sm;   // CTAs of this variant that fit on one SM
+  double efficiency;  // measured steady-state fraction of the arithmetic pipe's peak
   bool explicit_only;  // never chosen automatically (comparison variants)
 };
 
@@ -30,7 +31,7 @@ struct MachineRates {
 inline MachineRates machine_rates(int elem_bytes) {
   MachineRates r;
   r.fma_per_clk = elem_bytes == 8 ? 64.0 : 128.0;
-  r.l2_bytes_per_clk = 24.0;
+  r.l2_bytes_per_clk = 32.0;
   r.hbm_bytes_per_clk = 22.0;
   r.tile_fixed_clks = 4000.0;
   return r;
@@ -45,7 +46,7 @@ inline double estimate_clks(const TileChoice& c, int64_t m, int64_t n, int64_t k
   const double per_sm = (double)(int64_t)((tiles + sms - 1) / sms);
   const double fma_tile = (double)c.bm * c.bn * c.bk * kt;
   // arithmetic pipe
-  double t_math = fma_tile / r.fma_per_clk;
+  const double t_math = fma_tile / (r.fma_per_clk * c.efficiency);
   // feed: bytes of A and B a tile pulls through L2 per multiply-add
   const double feed_tile = (double)(c.bm + c.bn) * c.bk * kt * elem_bytes;
   const double t_feed = feed_tile / r.l2_bytes_per_clk;

@@ -21,6 +21,7 @@ KINDS = {
     "dmma_m16n8k4": 3,
     "dmma_m16n8k8": 4,
     "dmma_m16n8k16": 5,
+    "ffma2": 6,
 }
 
 
