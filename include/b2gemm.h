@@ -47,7 +47,8 @@ typedef enum {
   B2_ERR_TIMEOUT = 1001,   /* a bounded device-side wait gave up */
   B2_ERR_LAUNCH = 1002,    /* the CUDA runtime refused a launch or a copy */
   B2_ERR_WORKSPACE = 1003, /* workspace pointer null, misaligned or too small */
-  B2_ERR_VARIANT = 1004    /* unknown or inapplicable kernel variant */
+  B2_ERR_VARIANT = 1004,   /* unknown or inapplicable kernel variant */
+  B2_ERR_STATIC_LIMIT = 1005 /* problem needs more scratch than the built-in array of b2_zgemm4m_static holds */
 } b2_status;
 
 /* Kernel variants (micro-kernel x tile).  B2_VARIANT_AUTO lets the analytic selector choose. */
@@ -112,6 +113,34 @@ size_t b2_zgemm4m_workspace_bytes(char transa, char transb, int64_t m, int64_t n
 int b2_zgemm4m(char transa, char transb, int64_t m, int64_t n, int64_t k, const double alpha[2], const void* A,
                int64_t lda, const void* B, int64_t ldb, const double beta[2], void* C, int64_t ldc,
                void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * b2_zgemm4m for callers that cannot allocate device memory.  (The paper has no counterpart;
+ * this is a convenience of the library.)
+ *
+ * Some callers have no way to obtain a workspace: code that runs where cudaMalloc is off
+ * limits (inside a latency-critical loop that must not take the allocator's lock, in a
+ * plug-in whose host forbids allocation, after the application has handed all device memory
+ * to its own pool).  For them the six real planes of the 4M scheme live in a scratch array
+ * that is part of the library image: B2_ZGEMM4M_STATIC_BYTES bytes of device memory on every
+ * GPU that loads the library, held until the process exits.  The caller passes only the
+ * operands; same arguments, semantics and return values as b2_zgemm4m otherwise.
+ *
+ *   - Limit: b2_zgemm4m_workspace_bytes(transa, transb, m, n, k) must not exceed
+ *     B2_ZGEMM4M_STATIC_BYTES (6 MiB: e.g. m = n = k = 256 needs 3 MiB, 360^3 just fits).
+ *     Larger problems return B2_ERR_STATIC_LIMIT and launch nothing.
+ *   - The call allocates and frees nothing, neither directly nor through a library.
+ *   - The first call on each device looks up the array's device address (the device must be
+ *     current); make that first call outside any stream capture.
+ *   - All calls on a device share the one array, and it keeps the previous call's contents.
+ *     Nothing in it has to start at zero (every plane element is written before it is read
+ *     within a call), but two calls that overlap on the GPU -- different streams, or
+ *     different host threads -- race on it: serialise them.
+ */
+#define B2_ZGEMM4M_STATIC_BYTES (6u << 20)
+int b2_zgemm4m_static(char transa, char transb, int64_t m, int64_t n, int64_t k, const double alpha[2],
+                      const void* A, int64_t lda, const void* B, int64_t ldb, const double beta[2], void* C,
+                      int64_t ldc, void* cuda_stream);
 
 /*
  * Host-buffer forms: A, B, C are HOST pointers (pinned memory makes the copies asynchronous),

@@ -34,6 +34,8 @@ _SIGNATURES = {
     "b2_zgemm4m": (c_int, [c_char, c_char, c_int64, c_int64, c_int64, ctypes.POINTER(c_double), c_void_p, c_int64,
                            c_void_p, c_int64, ctypes.POINTER(c_double), c_void_p, c_int64, c_void_p, c_size_t,
                            c_void_p]),
+    "b2_zgemm4m_static": (c_int, [c_char, c_char, c_int64, c_int64, c_int64, ctypes.POINTER(c_double), c_void_p, c_int64,
+                                  c_void_p, c_int64, ctypes.POINTER(c_double), c_void_p, c_int64, c_void_p]),
     "b2_gemm_host_workspace_bytes": (c_size_t, [c_int, c_char, c_char, c_int64, c_int64, c_int64]),
     "b2_dgemm_host": (c_int, _GEMM_TAIL_D + [c_void_p, c_size_t, c_void_p]),
     "b2_sgemm_host": (c_int, _GEMM_TAIL_S + [c_void_p, c_size_t, c_void_p]),
@@ -157,6 +159,26 @@ def b2_zgemm4m(transa, transb, m, n, k, alpha, A, lda, B, ldb, beta, C, ldc, wor
                           _ptr(workspace), wbytes, _stream())
     if check:
         _check("b2_zgemm4m", rc)
+    return rc
+
+
+ZGEMM4M_STATIC_BYTES = 6 << 20
+
+
+def b2_zgemm4m_static(transa, transb, m, n, k, alpha, A, lda, B, ldb, beta, C, ldc, check=True) -> int:
+    """b2_zgemm4m without a workspace argument, for callers that cannot allocate device memory.
+
+    The scratch planes live in a ZGEMM4M_STATIC_BYTES array inside the library; problems that need more
+    return B2_ERR_STATIC_LIMIT (1005).  Calls share that array: do not overlap them on the GPU."""
+    for t in (A, B, C):
+        if t is not None and (t.dtype != torch.complex128 or not t.is_cuda):
+            raise TypeError("b2_zgemm4m_static takes complex128 CUDA tensors")
+    al = (c_double * 2)(complex(alpha).real, complex(alpha).imag)
+    be = (c_double * 2)(complex(beta).real, complex(beta).imag)
+    rc = lib().b2_zgemm4m_static(_tr(transa), _tr(transb), m, n, k, al, _ptr(A), lda, _ptr(B), ldb, be, _ptr(C), ldc,
+                                 _stream())
+    if check:
+        _check("b2_zgemm4m_static", rc)
     return rc
 
 

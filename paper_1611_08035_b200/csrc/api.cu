@@ -231,6 +231,7 @@ extern "C" const char* b2_strerror(int status) {
     case B2_ERR_LAUNCH: return "CUDA launch or copy failed";
     case B2_ERR_WORKSPACE: return "workspace or output buffer null, misaligned or too small";
     case B2_ERR_VARIANT: return "unknown or inapplicable kernel variant";
+    case B2_ERR_STATIC_LIMIT: return "problem needs more scratch than the built-in array of b2_zgemm4m_static holds";
     case -1: return "argument 1 is illegal";
     case -2: return "argument 2 is illegal";
     case -3: return "argument 3 is illegal";

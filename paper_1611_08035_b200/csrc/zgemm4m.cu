@@ -154,3 +154,28 @@ extern "C" int b2_zgemm4m(char transa, char transb, int64_t m, int64_t n, int64_
   zmerge_kernel<<<grid_for(m * n), 256, 0, st>>>(m, n, Cr, Ci, p.lpc, Cz, ldc);
   return cudaGetLastError() == cudaSuccess ? B2_OK : B2_ERR_LAUNCH;
 }
+
+// ---- b2_zgemm4m without a caller-provided workspace -------------------------------------------
+// The scratch planes live in the library image.  In host code the array's name is only a
+// host-side stand-in for the symbol, not a device address: the address each device maps it
+// to is looked up once per device with cudaGetSymbolAddress and cached.
+static __device__ __align__(256) unsigned char g_zgemm4m_scratch[B2_ZGEMM4M_STATIC_BYTES];
+
+extern "C" int b2_zgemm4m_static(char transa, char transb, int64_t m, int64_t n, int64_t k, const double alpha[2],
+                                 const void* A, int64_t lda, const void* B, int64_t ldb, const double beta[2],
+                                 void* C, int64_t ldc, void* cuda_stream) {
+  using namespace b2;
+  static void* scratch_by_device[64] = {};
+  if ((is_n(transa) || is_t(transa)) && (is_n(transb) || is_t(transb)) && m >= 0 && n >= 0 && k >= 0 &&
+      make_plan(transa, transb, m, n, k).total > (size_t)B2_ZGEMM4M_STATIC_BYTES)
+    return B2_ERR_STATIC_LIMIT;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return B2_ERR_LAUNCH;
+  if (!scratch_by_device[dev]) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_zgemm4m_scratch) != cudaSuccess || !ptr) return B2_ERR_LAUNCH;
+    scratch_by_device[dev] = ptr;
+  }
+  return b2_zgemm4m(transa, transb, m, n, k, alpha, A, lda, B, ldb, beta, C, ldc, scratch_by_device[dev],
+                    (size_t)B2_ZGEMM4M_STATIC_BYTES, cuda_stream);
+}
