@@ -93,8 +93,33 @@ struct Stager {
     }
   }
 
-  // General path.  X0 points at element (o0, k0) of the operand; o_valid / k_valid are the numbers of valid
-  // rows and k-entries from there.
+  // Edge tile, full slab: only o_valid (< BO) rows/columns of the tile exist.  Chunks that lie entirely outside
+  // are skipped, not zero-filled: whatever the shared-memory rows beyond o_valid hold only feeds accumulators of
+  // rows/columns >= m or n of C, which the epilogue never stores.  A chunk that straddles the edge copies its
+  // valid bytes only.  No address outside the operand is formed into a load.
+  __device__ __forceinline__ void load_edge(T* __restrict__ s, int o_valid, int tid) const {
+#pragma unroll
+    for (int it = 0; it < ITER; ++it) {
+      if constexpr (STRAIGHT) {
+        if constexpr (SRC == OC) {  // chunk runs along o; every line (k) is valid
+          const int nvalid = o_valid - (tid % CPL) * VEC;
+          if (nvalid > 0)
+            cp_async_zfill<VEC * ELEM>(s + dst0 + it * LSTEP * PITCH, src + it * lstep,
+                                       (nvalid < VEC ? nvalid : VEC) * ELEM);
+        } else {  // lines are o-rows; chunk runs along k (all valid)
+          if (tid / CPL + it * LSTEP < o_valid)
+            cp_async_zfill<VEC * ELEM>(s + dst0 + it * LSTEP * PITCH, src + it * lstep, VEC * ELEM);
+        }
+      } else {
+        const int a = it % Q, b = it / Q;
+        if (tid / RUN + a * LSTEP < o_valid)
+          cp_async_zfill<ELEM>(s + dst0 + b * RUN * PITCH + a * LSTEP, src + a * lstep + b * RUN, ELEM);
+      }
+    }
+  }
+
+  // General path (partial k-slab).  X0 points at element (o0, k0) of the operand; o_valid / k_valid are the
+  // numbers of valid rows and k-entries from there; everything beyond is zero-filled.
   static __device__ __noinline__ void load_general(T* __restrict__ s, const T* __restrict__ X0, int64_t ld,
                                                    int o_valid, int k_valid, int tid) {
     if constexpr (STRAIGHT) {
@@ -524,14 +549,19 @@ struct GemmKernel {
       const int k_valid = (kt == KT - 1) ? k_tail : BK;
       T* dA = sA + slot * Micro::A_STAGE;
       T* dB = sB + slot * Micro::B_STAGE;
-      if (a_inside && k_valid == BK) {
-        stA.load_fast(dA);
+      if (k_valid == BK) {
+        if (a_inside) {
+          stA.load_fast(dA);
+        } else {
+          stA.load_edge(dA, m_valid, tid);
+        }
+        if (b_inside) {
+          stB.load_fast(dB);
+        } else {
+          stB.load_edge(dB, n_valid, tid);
+        }
       } else {
         StageA::load_general(dA, gA + kt * stepA, p.lda, m_valid, k_valid, tid);
-      }
-      if (b_inside && k_valid == BK) {
-        stB.load_fast(dB);
-      } else {
         StageB::load_general(dB, gB + kt * stepB, p.ldb, n_valid, k_valid, tid);
       }
       stA.advance();
