@@ -177,6 +177,33 @@ int b2_sgemm_host(char transa, char transb, int64_t m, int64_t n, int64_t k, flo
 int b2_pipe_probe(int kind, int threads_per_cta, int ctas, int64_t iters, void* scratch, size_t scratch_bytes,
                   double* fma_per_thread_iter, void* cuda_stream);
 
+/*
+ * The paper's analytical model (host-only calls; nothing is launched, no GPU is needed).
+ *
+ * b2_model_throughput: Section 4 ("Little's Law").  Pipelines i = 0..npipes-1 retire rate[i]
+ *   instructions per cycle; an instruction mix puts jobs[i] instructions on pipeline i per outer
+ *   product.  Returns outer products per cycle = min_i rate[i] / jobs[i] over pipelines with
+ *   jobs[i] > 0 (infinity when there is none), or -1 for invalid input (npipes <= 0, null
+ *   pointers, rate <= 0, jobs < 0).  rate and jobs are HOST arrays.
+ * b2_model_stalled_throughput: Section 4 ("Estimating throughput").  A pipeline whose n_dependent
+ *   instructions of latency `latency` cannot be overlapped needs W = jobs + n_dependent*latency
+ *   cycles; returns 1/W, or -1 for invalid input.
+ * b2_model_register_updates: Section 5 ("Limits imposed by registers").  Stores
+ *   floor((r_total - mr*nr/v - r_a) / r_r) in *n_updates (HOST); returns 0, -1 for non-positive
+ *   sizes, -7 for a null output.
+ * b2_model_predict_variant: the Section 4 estimate applied to one sub-partition of a B200 SM
+ *   (pipelines: issue, FP64 FMA, FP64 tensor, FP32 FMA, shared-memory wavefronts; rates from
+ *   b2_pipe_probe) for kernel variant `variant` of `dtype`.  Stores the predicted fraction of the
+ *   arithmetic pipe's peak in *fraction and, when json_out is not NULL, a JSON object with the
+ *   jobs per pipeline per rank-1 update, the clocks each pipeline needs, the prediction and the
+ *   measured steady-state fraction (HOST buffer of cap bytes).  Returns 0, -1/-2/-3 for a bad
+ *   dtype / variant / null fraction, B2_ERR_WORKSPACE when cap is too small.
+ */
+double b2_model_throughput(int npipes, const double* rate, const double* jobs);
+double b2_model_stalled_throughput(double jobs, int n_dependent, double latency);
+int b2_model_register_updates(int r_total, int mr, int nr, int v, int r_a, int r_r, int* n_updates);
+int b2_model_predict_variant(int dtype, int variant, double* fraction, char* json_out, size_t cap);
+
 /* Static, NUL-terminated text for a return value of any call above. */
 const char* b2_strerror(int status);
 /* Static, NUL-terminated library version. */

@@ -40,6 +40,10 @@ _SIGNATURES = {
     "b2_dgemm_host": (c_int, _GEMM_TAIL_D + [c_void_p, c_size_t, c_void_p]),
     "b2_sgemm_host": (c_int, _GEMM_TAIL_S + [c_void_p, c_size_t, c_void_p]),
     "b2_pipe_probe": (c_int, [c_int, c_int, c_int, c_int64, c_void_p, c_size_t, ctypes.POINTER(c_double), c_void_p]),
+    "b2_model_throughput": (c_double, [c_int, ctypes.POINTER(c_double), ctypes.POINTER(c_double)]),
+    "b2_model_stalled_throughput": (c_double, [c_double, c_int, c_double]),
+    "b2_model_register_updates": (c_int, [c_int, c_int, c_int, c_int, c_int, c_int, ctypes.POINTER(c_int)]),
+    "b2_model_predict_variant": (c_int, [c_int, c_int, ctypes.POINTER(c_double), c_char_p, c_size_t]),
     "b2_strerror": (c_char_p, [c_int]),
     "b2_version": (c_char_p, []),
 }
@@ -208,3 +212,32 @@ def b2_sgemm_host(transa, transb, m, n, k, alpha, A, lda, B, ldb, beta, C, ldc, 
     """b2_sgemm on HOST tensors (pinned for speed); copies in, computes on the GPU, copies C back."""
     return _host_call("b2_sgemm_host", torch.float32, transa, transb, m, n, k, alpha, A, lda, B, ldb, beta, C, ldc,
                       workspace, check)
+
+
+def b2_model_throughput(rates, jobs) -> float:
+    """Section 4: outer products per cycle of an instruction mix = min over pipelines of rate/jobs."""
+    n = len(rates)
+    if n != len(jobs):
+        raise ValueError("rates and jobs must have the same length")
+    r = (c_double * max(n, 1))(*rates)
+    j = (c_double * max(n, 1))(*jobs)
+    return lib().b2_model_throughput(n, r, j)
+
+
+def b2_model_stalled_throughput(jobs: float, n_dependent: int, latency: float) -> float:
+    return lib().b2_model_stalled_throughput(jobs, n_dependent, latency)
+
+
+def b2_model_register_updates(r_total, mr, nr, v, r_a, r_r) -> int:
+    """Section 5: floor((R_total - mr*nr/v - R_A) / R_R)."""
+    out = c_int(0)
+    _check("b2_model_register_updates", lib().b2_model_register_updates(r_total, mr, nr, v, r_a, r_r, ctypes.byref(out)))
+    return out.value
+
+
+def b2_model_predict_variant(dtype: int, variant: int):
+    """(predicted fraction of pipe peak, JSON description) of a kernel variant from the pipeline model."""
+    frac = c_double(0.0)
+    buf = ctypes.create_string_buffer(1024)
+    _check("b2_model_predict_variant", lib().b2_model_predict_variant(dtype, variant, ctypes.byref(frac), buf, len(buf)))
+    return frac.value, buf.value.decode()

@@ -18,6 +18,7 @@ int launch_f64_v3(const GemmArgs<double>&, bool, bool, bool, cudaStream_t);
 int launch_f32_v0(const GemmArgs<float>&, bool, bool, bool, cudaStream_t);
 int launch_f32_v1(const GemmArgs<float>&, bool, bool, bool, cudaStream_t);
 int launch_f32_v2(const GemmArgs<float>&, bool, bool, bool, cudaStream_t);
+int launch_f32_v3(const GemmArgs<float>&, bool, bool, bool, cudaStream_t);
 
 namespace {
 
@@ -30,11 +31,12 @@ const VariantInfo kF64Info[] = {
 };
 const LaunchFn<double> kF64Launch[] = {launch_f64_v0, launch_f64_v1, launch_f64_v2, launch_f64_v3};
 const VariantInfo kF32Info[] = {
-    {"ffma_128x128x16_s4", "ffma", 128, 128, 16, 4, 256, 2, 0.72},
-    {"ffma_128x64x16_s4", "ffma", 128, 64, 16, 4, 128, 4, 0.75},
-    {"ffma_64x64x16_s4", "ffma", 64, 64, 16, 4, 64, 8, 0.68},
+    {"ffma2_128x128x16_s4", "ffma2", 128, 128, 16, 4, 256, 2, 0.72},
+    {"ffma2_128x64x16_s4", "ffma2", 128, 64, 16, 4, 128, 4, 0.75},
+    {"ffma2_64x64x16_s4", "ffma2", 64, 64, 16, 4, 64, 8, 0.68},
+    {"ffma_128x64x16_s4", "ffma", 128, 64, 16, 4, 128, 4, 0.70},
 };
-const LaunchFn<float> kF32Launch[] = {launch_f32_v0, launch_f32_v1, launch_f32_v2};
+const LaunchFn<float> kF32Launch[] = {launch_f32_v0, launch_f32_v1, launch_f32_v2, launch_f32_v3};
 
 }  // namespace
 
@@ -111,7 +113,7 @@ int choose_variant(int64_t m, int64_t n, int64_t k) {
   TileChoice cand[16];
   for (int v = 0; v < count && v < 16; ++v) {
     const VariantInfo& vi = variant_info_t<T>(v);
-    cand[v] = TileChoice{vi.bm, vi.bn, vi.bk, vi.threads, vi.ctas_per_sm, vi.efficiency, strcmp(vi.micro, "dfma") == 0};
+    cand[v] = TileChoice{vi.bm, vi.bn, vi.bk, vi.threads, vi.ctas_per_sm, vi.efficiency, strcmp(vi.micro, "dfma") == 0 || strcmp(vi.micro, "ffma") == 0};
   }
   return select_tile(cand, count < 16 ? count : 16, m, n, k, sm_count_cached(), (int)sizeof(T));
 }

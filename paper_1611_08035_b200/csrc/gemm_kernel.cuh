@@ -309,9 +309,11 @@ struct DmmaMicro {
 // 16-byte shared-memory loads: 64 independent FMAs per outer product.
 // A warp is 8 lanes along m by 4 lanes along n, so it covers 64 x 32 of C.
 // ---------------------------------------------------------------------------------------
-template <typename T_, int BM_, int BN_, int BK_, int WARPS_M, int WARPS_N, bool TA, bool TB>
+template <typename T_, int BM_, int BN_, int BK_, int WARPS_M, int WARPS_N, bool TA, bool TB, bool PACKED = true>
 struct SimtMicro {
   using T = T_;
+  // fp32 only: PACKED uses the pair instruction fma.rn.f32x2; false keeps scalar FFMA (comparison variant)
+  static constexpr bool PAIRS = (sizeof(T_) == 4) && PACKED;
   static constexpr int BM = BM_, BN = BN_, BK = BK_;
   static constexpr int NT = 32 * WARPS_M * WARPS_N;
   static constexpr int VEC = 16 / sizeof(T);
@@ -330,10 +332,10 @@ struct SimtMicro {
   struct AccPairs {
     unsigned long long p[TM / 2][TN];
   };
-  using Acc = typename std::conditional<sizeof(T) == 4, AccPairs, AccScalar>::type;
+  using Acc = typename std::conditional<PAIRS, AccPairs, AccScalar>::type;
 
   static __device__ __forceinline__ void zero(Acc& acc) {
-    if constexpr (sizeof(T) == 4) {
+    if constexpr (PAIRS) {
 #pragma unroll
       for (int i = 0; i < TM / 2; ++i)
 #pragma unroll
@@ -348,7 +350,7 @@ struct SimtMicro {
 
   // accumulator element (i, j)
   static __device__ __forceinline__ T get(const Acc& acc, int i, int j) {
-    if constexpr (sizeof(T) == 4) {
+    if constexpr (PAIRS) {
       float lo, hi;
       asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(acc.p[i / 2][j]));
       return (i & 1) ? hi : lo;
@@ -371,7 +373,7 @@ struct SimtMicro {
     const int lx = lane & 7, ly = lane >> 3;
     const T* pa = sA + warp_m * WTM + lx * VEC;
     const T* pb = sB + warp_n * WTN + ly * VEC;
-    if constexpr (sizeof(T) == 4) {
+    if constexpr (PAIRS) {
       // FP32: packed pair multiply-adds (fma.rn.f32x2, two IEEE fp32 FMAs per instruction).  A pair holds two
       // adjacent rows of one column of the accumulator block; a is used pairwise as loaded, b is duplicated
       // into both halves.  32 instructions instead of 64 per outer product: the FP32 pipe stays busy while

@@ -97,7 +97,7 @@ def test_selector_is_sane_without_gpu(b2):
         assert cfg["grid"] == cfg["tiles_m"] * cfg["tiles_n"]
     assert tiny["BM"] * tiny["BN"] <= 64 * 64
     f32 = json.loads(b2.b2_gemm_query_config(1, "N", "T", 4096, 4096, 4096, 4096, 4096, 4096))
-    assert f32["micro_kernel"] == "ffma" and f32["dtype"] == "f32"
+    assert f32["micro_kernel"] == "ffma2" and f32["dtype"] == "f32"
     with pytest.raises(b2.B2Error):
         b2.b2_gemm_query_config(0, "N", "N", 8, 8, 8, 4, 8, 8)
     with pytest.raises(b2.B2Error):

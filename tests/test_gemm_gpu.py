@@ -254,7 +254,7 @@ def test_query_config_reports_launch(b2):
     assert cfg["micro_kernel"] == "dmma" and cfg["grid"] == cfg["tiles_m"] * cfg["tiles_n"]
     assert cfg["tiles_m"] == -(-8192 // cfg["BM"]) and cfg["k_slabs"] == 8192 // cfg["kc"]
     cfg = json.loads(b2.b2_gemm_query_config(1, "T", "N", 1001, 999, 1003, 1027, 1027, 1027))
-    assert cfg["micro_kernel"] == "ffma" and cfg["vector_staging_if_pointers_aligned"] is False
+    assert cfg["micro_kernel"] == "ffma2" and cfg["vector_staging_if_pointers_aligned"] is False
 
 
 def test_pipe_probe_rates(b2):
