@@ -79,6 +79,22 @@ int b2_sgemm_variant(int variant, char transa, char transb, int64_t m, int64_t n
                      const float* A, int64_t lda, const float* B, int64_t ldb, float beta, float* C,
                      int64_t ldc, void* cuda_stream);
 
+/*
+ * Device-side status.  Kernels that wait on hardware barriers (the TMA-staged variants) bound
+ * every wait; when a bound is hit they record B2_ERR_TIMEOUT in a status word on the device,
+ * stop computing and return, leaving C unspecified.  b2_device_status synchronises `cuda_stream`,
+ * returns that word (B2_OK when nothing happened) and clears it; B2_ERR_LAUNCH when the
+ * synchronisation or the copy fails.  It is the only call of this library that blocks besides
+ * the host-buffer forms.
+ */
+int b2_device_status(void* cuda_stream);
+/*
+ * Self-test of that mechanism: enqueues a one-warp kernel that waits, with a bound of a few
+ * thousand polls, on a barrier nothing completes, so the next b2_device_status returns
+ * B2_ERR_TIMEOUT.  Nothing faults or hangs.  Returns 0 or B2_ERR_LAUNCH.
+ */
+int b2_selftest_wait_timeout(void* cuda_stream);
+
 /* dtype codes for the query calls */
 #define B2_F64 0
 #define B2_F32 1

@@ -26,6 +26,8 @@ _SIGNATURES = {
     "b2_sgemm": (c_int, _GEMM_TAIL_S + [c_void_p]),
     "b2_dgemm_variant": (c_int, [c_int] + _GEMM_TAIL_D + [c_void_p]),
     "b2_sgemm_variant": (c_int, [c_int] + _GEMM_TAIL_S + [c_void_p]),
+    "b2_device_status": (c_int, [c_void_p]),
+    "b2_selftest_wait_timeout": (c_int, [c_void_p]),
     "b2_variant_count": (c_int, [c_int]),
     "b2_variant_name": (c_char_p, [c_int, c_int]),
     "b2_gemm_query_config": (c_int, [c_int, c_char, c_char, c_int64, c_int64, c_int64, c_int64, c_int64, c_int64,
@@ -241,3 +243,13 @@ def b2_model_predict_variant(dtype: int, variant: int):
     buf = ctypes.create_string_buffer(1024)
     _check("b2_model_predict_variant", lib().b2_model_predict_variant(dtype, variant, ctypes.byref(frac), buf, len(buf)))
     return frac.value, buf.value.decode()
+
+
+def b2_device_status() -> int:
+    """Synchronise the current stream and return (and clear) the device status word: 0 or B2_ERR_TIMEOUT."""
+    return lib().b2_device_status(_stream())
+
+
+def b2_selftest_wait_timeout() -> int:
+    """Enqueue the bounded-wait self-test kernel (the next b2_device_status then reports B2_ERR_TIMEOUT)."""
+    return lib().b2_selftest_wait_timeout(_stream())

@@ -15,6 +15,9 @@ int launch_f64_v0(const GemmArgs<double>&, bool, bool, bool, cudaStream_t);
 int launch_f64_v1(const GemmArgs<double>&, bool, bool, bool, cudaStream_t);
 int launch_f64_v2(const GemmArgs<double>&, bool, bool, bool, cudaStream_t);
 int launch_f64_v3(const GemmArgs<double>&, bool, bool, bool, cudaStream_t);
+int launch_f64_v4(const GemmArgs<double>&, bool, bool, bool, cudaStream_t);
+int launch_f64_v5(const GemmArgs<double>&, bool, bool, bool, cudaStream_t);
+int launch_f64_v6(const GemmArgs<double>&, bool, bool, bool, cudaStream_t);
 int launch_f32_v0(const GemmArgs<float>&, bool, bool, bool, cudaStream_t);
 int launch_f32_v1(const GemmArgs<float>&, bool, bool, bool, cudaStream_t);
 int launch_f32_v2(const GemmArgs<float>&, bool, bool, bool, cudaStream_t);
@@ -28,8 +31,12 @@ const VariantInfo kF64Info[] = {
     {"dmma_128x64x16_s3", "dmma", 128, 64, 16, 3, 128, 2, 0.94},
     {"dmma_64x64x16_s3", "dmma", 64, 64, 16, 3, 128, 4, 0.955},
     {"dfma_128x64x16_s3", "dfma", 128, 64, 16, 3, 128, 2, 0.73},
+    {"dmma_tma_64x64x16_s3", "dmma_tma", 64, 64, 16, 3, 128, 4, 0.97},
+    {"dmma_tma_128x64x16_s3", "dmma_tma", 128, 64, 16, 3, 128, 2, 0.945},
+    {"dmma_tma_128x128x16_s4", "dmma_tma", 128, 128, 16, 4, 256, 1, 0.95},
 };
-const LaunchFn<double> kF64Launch[] = {launch_f64_v0, launch_f64_v1, launch_f64_v2, launch_f64_v3};
+const LaunchFn<double> kF64Launch[] = {launch_f64_v0, launch_f64_v1, launch_f64_v2, launch_f64_v3,
+                                       launch_f64_v4, launch_f64_v5, launch_f64_v6};
 const VariantInfo kF32Info[] = {
     {"ffma2_128x128x16_s4", "ffma2", 128, 128, 16, 4, 256, 2, 0.72},
     {"ffma2_128x64x16_s4", "ffma2", 128, 64, 16, 4, 128, 4, 0.75},
@@ -107,13 +114,17 @@ static bool operands_aligned(const T* A, int64_t lda, const T* B, int64_t ldb) {
          (lda % VEC == 0) && (ldb % VEC == 0);
 }
 
+// `aligned`: A and B have 16-byte aligned columns, which the TMA-staged variants need.
 template <typename T>
-int choose_variant(int64_t m, int64_t n, int64_t k) {
+int choose_variant(int64_t m, int64_t n, int64_t k, bool aligned) {
   const int count = variant_count_t<T>();
   TileChoice cand[16];
   for (int v = 0; v < count && v < 16; ++v) {
     const VariantInfo& vi = variant_info_t<T>(v);
-    cand[v] = TileChoice{vi.bm, vi.bn, vi.bk, vi.threads, vi.ctas_per_sm, vi.efficiency, strcmp(vi.micro, "dfma") == 0 || strcmp(vi.micro, "ffma") == 0};
+    const bool comparison_only = strcmp(vi.micro, "dfma") == 0 || strcmp(vi.micro, "ffma") == 0;
+    const bool needs_alignment = strcmp(vi.micro, "dmma_tma") == 0;
+    cand[v] = TileChoice{vi.bm, vi.bn, vi.bk, vi.threads, vi.ctas_per_sm, vi.efficiency,
+                         comparison_only || (needs_alignment && !aligned)};
   }
   return select_tile(cand, count < 16 ? count : 16, m, n, k, sm_count_cached(), (int)sizeof(T));
 }
@@ -137,7 +148,7 @@ int gemm_entry(int variant, char transa, char transb, int64_t m, int64_t n, int6
     scale_kernel<T><<<(unsigned)blocks, threads, 0, stream>>>(m, n, beta, C, ldc);
     return cudaGetLastError() == cudaSuccess ? B2_OK : B2_ERR_LAUNCH;
   }
-  if (variant == B2_VARIANT_AUTO) variant = choose_variant<T>(m, n, k);
+  if (variant == B2_VARIANT_AUTO) variant = choose_variant<T>(m, n, k, operands_aligned(A, lda, B, ldb));
   GemmArgs<T> args;
   args.m = m, args.n = n, args.k = k;
   args.alpha = alpha, args.beta = beta;
@@ -205,11 +216,12 @@ extern "C" int b2_gemm_query_config(int dtype, char transa, char transb, int64_t
   const int bad = b2::check_gemm_args(transa, transb, m, n, k, dummy, lda, dummy, ldb, dummy, ldc, true);
   if (bad) return bad - 1;
   if (!json_out) return -11;
-  const int v = dtype == B2_F64 ? b2::choose_variant<double>(m, n, k) : b2::choose_variant<float>(m, n, k);
-  const b2::VariantInfo& vi = dtype == B2_F64 ? b2::f64_variant_info(v) : b2::f32_variant_info(v);
-  const long long tiles_m = (m + vi.bm - 1) / vi.bm, tiles_n = (n + vi.bn - 1) / vi.bn;
   const int elem = dtype == B2_F64 ? 8 : 4;
   const bool ld_aligned = (lda % (16 / elem) == 0) && (ldb % (16 / elem) == 0);
+  const int v = dtype == B2_F64 ? b2::choose_variant<double>(m, n, k, ld_aligned)
+                                : b2::choose_variant<float>(m, n, k, ld_aligned);
+  const b2::VariantInfo& vi = dtype == B2_F64 ? b2::f64_variant_info(v) : b2::f32_variant_info(v);
+  const long long tiles_m = (m + vi.bm - 1) / vi.bm, tiles_n = (n + vi.bn - 1) / vi.bn;
   char buf[768];
   const int len = snprintf(
       buf, sizeof(buf),

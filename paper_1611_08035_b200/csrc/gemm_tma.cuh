@@ -1,0 +1,183 @@
+// The fp64 tensor-core GEMM kernel with TMA staging: the same tile loop, micro-kernel and
+// epilogue as gemm_kernel.cuh, but the operand slabs are brought into shared memory by the
+// tensor memory accelerator (cp.async.bulk.tensor) and handed from producer to consumers
+// through mbarriers instead of cp.async groups and a CTA-wide barrier per slab.
+//
+// Why it fits: the DMMA micro-kernel reads either shared-memory layout, and both layouts are
+// dense boxes whose inner extent is the tile extent plus a few elements of padding (pitch =
+// 4 or 2 mod 16 doubles keeps every fragment load bank-conflict free).  So one TMA box per
+// operand per slab, with an inner extent of pitch elements, reproduces the staged tile exactly;
+// the few extra elements it fetches belong to the neighbouring tile and are never read.  TMA
+// zero-fills whatever lies outside the matrix, which covers edge tiles and the partial last
+// k-slab with no extra code (the paper's "packing" step, Section 2.1, done by hardware).
+//
+// Requirements (checked on the host): A and B 16-byte aligned with even leading dimensions.
+// Every wait on an mbarrier is bounded; when a bound is hit the kernel records
+// B2_ERR_TIMEOUT in a status word, stops computing, waits (bounded) for the copies it still
+// has in flight and returns.
+#pragma once
+#include <cuda.h>
+
+#include "gemm_kernel.cuh"
+
+namespace b2 {
+
+// ---- mbarrier / TMA primitives -------------------------------------------------------------
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_fence_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t done;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(done)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return done != 0;
+}
+// Bounded wait: false when the phase did not complete within kSpinLimit polls.
+constexpr uint32_t kSpinLimit = 1u << 24;
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, uint32_t limit = kSpinLimit) {
+  for (uint32_t spin = 0; spin < limit; ++spin)
+    if (mbar_try_wait(bar, parity)) return true;
+  return false;
+}
+// One 2-D box from global (through the tensor map) to shared memory, completion counted on `bar`.
+__device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* map, int c_inner, int c_outer,
+                                            uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(smem_u32(smem_dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(c_inner), "r"(c_outer),
+      "r"(smem_u32(bar))
+      : "memory");
+}
+
+// ---- the kernel ------------------------------------------------------------------------------
+template <class Micro, int STAGES, bool TA, bool TB>
+struct GemmTmaKernel {
+  using T = double;
+  static_assert(std::is_same<typename Micro::T, double>::value, "TMA staging is instantiated for the fp64 DMMA kernels");
+  static constexpr int BM = Micro::BM, BN = Micro::BN, BK = Micro::BK, NT = Micro::NT;
+  static constexpr int NWARPS = NT / 32;
+  // boxes: inner extent = shared-memory pitch, outer extent = number of lines of the staged tile
+  static constexpr int A_INNER = Micro::PA, A_OUTER = TA ? BM : BK;
+  static constexpr int B_INNER = Micro::PB, B_OUTER = TB ? BK : BN;
+  static_assert(A_INNER * A_OUTER == Micro::A_STAGE && B_INNER * B_OUTER == Micro::B_STAGE, "boxes tile the stages");
+  static constexpr uint32_t A_BYTES = Micro::A_STAGE * 8, B_BYTES = Micro::B_STAGE * 8;
+  static_assert(A_BYTES % 128 == 0 && B_BYTES % 128 == 0, "stages must keep 128-byte alignment");
+  static constexpr size_t SMEM_BYTES = (size_t)STAGES * (A_BYTES + B_BYTES) + 2 * STAGES * sizeof(uint64_t);
+
+  static __device__ __forceinline__ void run(const GemmArgs<T>& p, const CUtensorMap* mapA, const CUtensorMap* mapB,
+                                             int* status) {
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    T* sA = reinterpret_cast<T*>(smem_raw);
+    T* sB = sA + STAGES * Micro::A_STAGE;
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem_raw + (size_t)STAGES * (A_BYTES + B_BYTES));
+    uint64_t* empty = full + STAGES;
+
+    const int tid = threadIdx.x;
+    const int warp = tid >> 5, lane = tid & 31;
+    const int warp_m = warp % (BM / Micro::WTM), warp_n = warp / (BM / Micro::WTM);
+
+    int tm, tn;
+    tile_coords(blockIdx.x, p.tiles_m, p.tiles_n, p.group_m, tm, tn);
+    const int64_t m0 = (int64_t)tm * BM, n0 = (int64_t)tn * BN;
+    const int KT = (int)((p.k + BK - 1) / BK);
+
+    if (tid == 0) {
+      for (int s = 0; s < STAGES; ++s) {
+        mbar_init(&full[s], 1);        // one arrival (the producer's expect_tx) plus the bytes of both boxes
+        mbar_init(&empty[s], NWARPS);  // one arrival per consumer warp
+      }
+      mbar_fence_init();
+    }
+    __syncthreads();
+
+    // producer (thread 0): slab kt goes to slot kt % STAGES
+    auto issue = [&](int kt) {
+      const int slot = kt % STAGES;
+      const int k0 = kt * BK;
+      mbar_arrive_expect_tx(&full[slot], A_BYTES + B_BYTES);
+      tma_load_2d(sA + slot * Micro::A_STAGE, mapA, TA ? k0 : (int)m0, TA ? (int)m0 : k0, &full[slot]);
+      tma_load_2d(sB + slot * Micro::B_STAGE, mapB, TB ? (int)n0 : k0, TB ? k0 : (int)n0, &full[slot]);
+    };
+
+    int issued = 0;  // slabs handed to the TMA so far (thread 0 only)
+    if (tid == 0) {
+      for (; issued < STAGES - 1 && issued < KT; ++issued) issue(issued);
+    }
+
+    // beta != 0: pull the tile's old C values towards L2 while the k-loop runs
+    if (p.beta != T(0)) {
+      const int m_valid = (int)min((int64_t)BM, p.m - m0), n_valid = (int)min((int64_t)BN, p.n - n0);
+      constexpr int LINE = 16, LPC = (BM + LINE - 1) / LINE;
+      for (int c = tid; c < BN * LPC; c += NT) {
+        const int col = c / LPC, row = (c % LPC) * LINE;
+        if (col < n_valid && row < m_valid) {
+          const T* ptr = p.C + (n0 + col) * p.ldc + m0 + row;
+          asm volatile("prefetch.global.L2 [%0];" ::"l"(ptr));
+        }
+      }
+    }
+
+    typename Micro::Acc acc;
+    Micro::zero(acc);
+
+    bool ok = true;
+    int waited = 0;  // slabs whose arrival this thread has seen
+    for (int kt = 0; kt < KT; ++kt) {
+      const int slot = kt % STAGES;
+      // refill the slot that slab kt-1 used, once every warp has released it
+      if (tid == 0 && issued < KT) {
+        const int fslot = issued % STAGES;
+        const int round = issued / STAGES;  // how many times this slot has been filled before
+        if (round > 0 && !mbar_wait_bounded(&empty[fslot], (uint32_t)((round - 1) & 1))) {
+          ok = false;
+        } else {
+          issue(issued);
+          ++issued;
+        }
+      }
+      ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;  // thread 0's verdict reaches the rest of warp 0
+      if (!ok) break;
+      if (!mbar_wait_bounded(&full[slot], (uint32_t)((kt / STAGES) & 1))) {
+        ok = false;
+        break;
+      }
+      waited = kt + 1;
+      Micro::compute(acc, sA + slot * Micro::A_STAGE, sB + slot * Micro::B_STAGE, warp_m, warp_n, lane);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&empty[slot]);
+    }
+
+    if (!ok) {
+      // A bounded wait ran out: record it, let the copies still in flight land (their slots have not been
+      // refilled since, so the parity of their phase is unambiguous), and leave without storing anything.
+      atomicExch(status, (int)B2_ERR_TIMEOUT);
+      if (tid == 0) {
+        for (int kt = waited; kt < issued; ++kt)
+          (void)mbar_wait_bounded(&full[kt % STAGES], (uint32_t)((kt / STAGES) & 1));
+      }
+      return;
+    }
+    Micro::epilogue(acc, p, m0, n0, warp_m, warp_n, lane);
+  }
+};
+
+template <class Kernel, int MIN_CTAS>
+__global__ void __launch_bounds__(Kernel::NT, MIN_CTAS)
+    gemm_tma_kernel(const GemmArgs<double> p, const __grid_constant__ CUtensorMap mapA,
+                    const __grid_constant__ CUtensorMap mapB, int* status) {
+  Kernel::run(p, &mapA, &mapB, status);
+}
+
+}  // namespace b2

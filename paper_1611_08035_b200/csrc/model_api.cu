@@ -31,7 +31,7 @@ extern "C" int b2_model_predict_variant(int dtype, int variant, double* fraction
   if (!fraction) return -3;
   const VariantInfo& vi = dtype == B2_F64 ? f64_variant_info(variant) : f32_variant_info(variant);
   int kind;
-  if (strcmp(vi.micro, "dmma") == 0) kind = MK_DMMA;
+  if (strncmp(vi.micro, "dmma", 4) == 0) kind = MK_DMMA;
   else if (strcmp(vi.micro, "dfma") == 0) kind = MK_DFMA;
   else if (strcmp(vi.micro, "ffma2") == 0) kind = MK_FFMA2;
   else kind = MK_FFMA;

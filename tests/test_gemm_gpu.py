@@ -105,6 +105,35 @@ def test_all_variants_multi_tile_ragged(b2, oracle, kind):
                           expect_exact=True)
 
 
+def test_tma_variants_aligned_ragged_shapes(b2, oracle):
+    """The TMA-staged variants on shapes with ragged m, n and k (edge tiles and the partial last slab are
+    zero-filled by the hardware), even leading dimensions for A and B, an odd one for C."""
+    tma = [v for v in range(nvariants(b2, "d")) if "tma" in b2.b2_variant_name(0, v)]
+    assert len(tma) >= 3
+    for v in tma:
+        for ta, tb in TRANS:
+            for (m, n, k) in [(200, 136, 75), (129, 65, 17), (1, 1, 1), (7, 300, 33), (333, 270, 145), (64, 64, 1030)]:
+                (ra, _), (rb, _) = synth.operand_shapes(ta, tb, m, n, k)
+                lds = ((ra + 1) // 2 * 2 + 2, (rb + 1) // 2 * 2, m + (m + 1) % 2 + 0)
+                lds = (lds[0], lds[1], m | 1)
+                r = run_and_check(b2, oracle, "d", ta, tb, m, n, k, 0.7, -0.3, seed=m + k, variant=v, lds=lds)
+                assert r is not None
+                r = run_and_check(b2, oracle, "d", ta, tb, m, n, k, 1.5, 0.5, dist="int9", seed=m + k, variant=v,
+                                  lds=lds, expect_exact=True)
+                assert r is not None
+
+
+def test_bounded_wait_reports_timeout(b2):
+    """A device-side wait that nothing completes gives up after its bound and reports B2_ERR_TIMEOUT through the
+    status word; the context stays usable and the word is cleared by the read."""
+    assert b2.b2_device_status() == 0
+    assert b2.b2_selftest_wait_timeout() == 0
+    assert b2.b2_device_status() == 1001
+    assert b2.b2_device_status() == 0
+    x = torch.ones(8, device="cuda")
+    assert float(x.sum()) == 8.0
+
+
 @pytest.mark.parametrize("kind", ["d", "s"])
 def test_misaligned_base_pointers(b2, oracle, kind):
     """Base pointers shifted by one element (8- or 4-byte aligned only) with otherwise aligned leading dimensions."""
@@ -251,7 +280,9 @@ def test_host_entry_matches_oracle(b2, oracle, kind):
 def test_query_config_reports_launch(b2):
     import json
     cfg = json.loads(b2.b2_gemm_query_config(0, "N", "N", 8192, 8192, 8192, 8192, 8192, 8192))
-    assert cfg["micro_kernel"] == "dmma" and cfg["grid"] == cfg["tiles_m"] * cfg["tiles_n"]
+    assert cfg["micro_kernel"] == "dmma_tma" and cfg["grid"] == cfg["tiles_m"] * cfg["tiles_n"]
+    odd = json.loads(b2.b2_gemm_query_config(0, "N", "N", 1001, 999, 1003, 1027, 1027, 1027))
+    assert odd["micro_kernel"] == "dmma"
     assert cfg["tiles_m"] == -(-8192 // cfg["BM"]) and cfg["k_slabs"] == 8192 // cfg["kc"]
     cfg = json.loads(b2.b2_gemm_query_config(1, "T", "N", 1001, 999, 1003, 1027, 1027, 1027))
     assert cfg["micro_kernel"] == "ffma2" and cfg["vector_staging_if_pointers_aligned"] is False

@@ -136,6 +136,7 @@ def test_sm_predictions(b2):
     for name, (frac, d) in f64.items():
         bound = max(d["clocks_per_k"], key=d["clocks_per_k"].get)
         assert bound == ("tensor64" if name.startswith("dmma") else "fp64")
+    assert abs(pred["dmma_tma_64x64x16_s3"][1]["measured_fraction"] - 0.97) < 1e-9
     ffma = pred["ffma_128x64x16_s4"]
     ffma2 = pred["ffma2_128x64x16_s4"]
     assert max(ffma[1]["clocks_per_k"], key=ffma[1]["clocks_per_k"].get) == "issue"
