@@ -18,6 +18,8 @@ int launch_f64_v3(const GemmArgs<double>&, bool, bool, bool, cudaStream_t);
 int launch_f64_v4(const GemmArgs<double>&, bool, bool, bool, cudaStream_t);
 int launch_f64_v5(const GemmArgs<double>&, bool, bool, bool, cudaStream_t);
 int launch_f64_v6(const GemmArgs<double>&, bool, bool, bool, cudaStream_t);
+int launch_f64_t32(const GemmArgs<double>&, bool, bool, bool, cudaStream_t);
+int launch_f64_tma_t32(const GemmArgs<double>&, bool, bool, bool, cudaStream_t);
 int launch_f32_v0(const GemmArgs<float>&, bool, bool, bool, cudaStream_t);
 int launch_f32_v1(const GemmArgs<float>&, bool, bool, bool, cudaStream_t);
 int launch_f32_v2(const GemmArgs<float>&, bool, bool, bool, cudaStream_t);
@@ -34,9 +36,12 @@ const VariantInfo kF64Info[] = {
     {"dmma_tma_64x64x16_s3", "dmma_tma", 64, 64, 16, 3, 128, 4, 0.97},
     {"dmma_tma_128x64x16_s3", "dmma_tma", 128, 64, 16, 3, 128, 2, 0.945},
     {"dmma_tma_128x128x16_s4", "dmma_tma", 128, 128, 16, 4, 256, 1, 0.95},
+    {"dmma_32x32x16_s3", "dmma", 32, 32, 16, 3, 128, 6, 0.80},
+    {"dmma_tma_32x32x16_s3", "dmma_tma", 32, 32, 16, 3, 128, 6, 0.80},
 };
 const LaunchFn<double> kF64Launch[] = {launch_f64_v0, launch_f64_v1, launch_f64_v2, launch_f64_v3,
-                                       launch_f64_v4, launch_f64_v5, launch_f64_v6};
+                                       launch_f64_v4, launch_f64_v5, launch_f64_v6, launch_f64_t32,
+                                       launch_f64_tma_t32};
 const VariantInfo kF32Info[] = {
     {"ffma2_128x128x16_s4", "ffma2", 128, 128, 16, 4, 256, 2, 0.72},
     {"ffma2_128x64x16_s4", "ffma2", 128, 64, 16, 4, 128, 4, 0.75},

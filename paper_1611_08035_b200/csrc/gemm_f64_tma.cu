@@ -115,6 +115,8 @@ template <bool TA, bool TB>
 using MicroTma128x64 = DmmaMicro<128, 64, 16, 2, 2, TA, TB>;
 template <bool TA, bool TB>
 using MicroTma128 = DmmaMicro<128, 128, 16, 2, 4, TA, TB>;
+template <bool TA, bool TB>
+using MicroTmaT32 = DmmaMicro<32, 32, 16, 2, 2, TA, TB>;  // 4 warps of 16 x 16
 
 }  // namespace
 
@@ -126,6 +128,9 @@ int launch_f64_v5(const GemmArgs<double>& a, bool ta, bool tb, bool aligned, cud
 }
 int launch_f64_v6(const GemmArgs<double>& a, bool ta, bool tb, bool aligned, cudaStream_t s) {
   return launch_tma<MicroTma128, 4, 1>(a, ta, tb, aligned, s);
+}
+int launch_f64_tma_t32(const GemmArgs<double>& a, bool ta, bool tb, bool aligned, cudaStream_t s) {
+  return launch_tma<MicroTmaT32, 3, 6>(a, ta, tb, aligned, s);
 }
 
 }  // namespace b2
