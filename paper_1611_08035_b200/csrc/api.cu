@@ -44,7 +44,7 @@ const LaunchFn<double> kF64Launch[] = {launch_f64_v0, launch_f64_v1, launch_f64_
                                        launch_f64_tma_t32};
 const VariantInfo kF32Info[] = {
     {"ffma2_128x128x16_s4", "ffma2", 128, 128, 16, 4, 256, 2, 0.72},
-    {"ffma2_128x64x16_s4", "ffma2", 128, 64, 16, 4, 128, 4, 0.75},
+    {"ffma2_128x64x16_s4", "ffma2", 128, 64, 16, 4, 128, 3, 0.775},
     {"ffma2_64x64x16_s4", "ffma2", 64, 64, 16, 4, 64, 8, 0.68},
     {"ffma_128x64x16_s4", "ffma", 128, 64, 16, 4, 128, 4, 0.70},
 };

@@ -1,9 +1,9 @@
-// fp32 variant 1: FFMA outer products, 128 x 64 x 16 CTA tile, 4 warps, 4-stage ring, 4 CTAs/SM.
+// fp32 variant 1: FFMA outer products, 128 x 64 x 16 CTA tile, 4 warps, 4-stage ring, 3 CTAs/SM (168 registers: room to double-buffer the fragments).
 #include "gemm_launch.cuh"
 namespace b2 {
 template <bool TA, bool TB>
 using MicroF32V1 = SimtMicro<float, 128, 64, 16, 2, 2, TA, TB>;
 int launch_f32_v1(const GemmArgs<float>& a, bool ta, bool tb, bool aligned, cudaStream_t s) {
-  return VariantLauncher<MicroF32V1, 4, 4>::launch(a, ta, tb, aligned, s);
+  return VariantLauncher<MicroF32V1, 4, 3>::launch(a, ta, tb, aligned, s);
 }
 }  // namespace b2
