@@ -40,6 +40,12 @@ def lib() -> ctypes.CDLL:
                                                c_int64, c_void_p, c_int64]
         _lib.ref_zgemm_hi.argtypes = real_tail + [c_void_p, c_void_p, c_int64, c_void_p, c_int64, c_void_p, c_void_p,
                                                   c_int64, c_void_p, c_void_p, c_int64, c_void_p, c_int64]
+        _lib.ref_tf32_round.argtypes = [c_float]
+        _lib.ref_tf32_round.restype = c_float
+        _lib.ref_sgemm_tf32.argtypes = [c_int] + real_tail + [c_float, c_void_p, c_int64, c_void_p, c_int64, c_float,
+                                                              c_void_p, c_int64, c_void_p, c_void_p, c_int64, c_void_p,
+                                                              c_int64]
+        _lib.ref_sgemm_tf32.restype = c_int
         for fn in ("ref_dgemm", "ref_sgemm", "ref_dgemm_hi", "ref_sgemm_hi", "ref_zgemm", "ref_zgemm_hi",
                    "ref_num_threads"):
             getattr(_lib, fn).restype = c_int
@@ -176,3 +182,28 @@ def ref_zgemm_4m(transa, transb, m, n, k, alpha, A, lda, B, ldb, beta, C, ldc) -
         s = slice(j * ldc, j * ldc + m)
         Cv[0::2][s] = cr[s]
         Cv[1::2][s] = ci[s]
+
+
+def tf32_round(x: float) -> float:
+    """x (fp32) rounded to the nearest TF32 value (10 mantissa bits), ties away from zero."""
+    return float(lib().ref_tf32_round(float(np.float32(x))))
+
+
+def ref_sgemm_tf32(terms, transa, transb, m, n, k, alpha, A, lda, B, ldb, beta, C, ldc, cols=None):
+    """TF32 x1 (terms=1) or 3xTF32 (terms=3) GEMM by the definition, evaluated in double; returns (C_out fp32, S).
+
+    C is not modified.  C_out and S are flat with leading dimension max(1, m); columns outside `cols` are NaN."""
+    _flat(A, np.float32), _flat(B, np.float32), _flat(C, np.float32)
+    ldo = max(1, m)
+    out = np.full(ldo * max(n, 1), np.nan, dtype=np.float32)
+    S = np.full(ldo * max(n, 1), np.nan, dtype=np.float64)
+    if m > 0 and n > 0:
+        _check_storage(transa, transb, m, n, k, A, lda, B, ldb, C, ldc, True)
+    cptr, ncols, keep = _cols(cols)
+    rc = lib().ref_sgemm_tf32(terms, _tr(transa), _tr(transb), m, n, k, float(np.float32(alpha)), A.ctypes.data, lda,
+                              B.ctypes.data, ldb, float(np.float32(beta)), C.ctypes.data, ldc, out.ctypes.data,
+                              S.ctypes.data, ldo, cptr, ncols)
+    if rc != 0:
+        raise ValueError(f"oracle rejected argument {-rc}")
+    del keep
+    return out, S

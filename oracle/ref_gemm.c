@@ -235,3 +235,66 @@ int ref_num_threads(void) { return omp_get_max_threads(); }
 #else
 int ref_num_threads(void) { return 1; }
 #endif
+
+/*
+ * TF32 tensor-core variants of the fp32 GEMM (reported separately from the FP32-FMA entry; the paper has no
+ * counterpart, the definitions follow the published TF32 format: 1 sign, 8 exponent, 10 mantissa bits).
+ *
+ *   ref_tf32_round   x rounded to the nearest TF32 value, ties away from zero (the conversion the packing
+ *                    kernel applies, PTX cvt.rna.tf32.f32).
+ *   ref_sgemm_tf32   terms == 1:  acc_ij = sum_p t(a_ip) t(b_pj)                       ("TF32 x1")
+ *                    terms == 3:  a = ah + al with ah = t(a), al = t(a - ah) (likewise b),
+ *                                 acc_ij = sum_p (ah bh + ah bl + al bh)               ("3 x TF32")
+ *                    evaluated in double (every product of two TF32 values is exact in double), then
+ *                    Cout_ij = fp32(alpha*acc_ij + beta*C_ij), and S_ij = |alpha| sum_p |a_ip||b_pj| + |beta||C_ij|.
+ */
+float ref_tf32_round(float x) {
+  uint32_t u;
+  memcpy(&u, &x, 4);
+  if ((u & 0x7f800000u) == 0x7f800000u) return x; /* Inf, NaN unchanged */
+  u += 0x00001000u;                               /* half of the last kept place, magnitude-wise */
+  u &= 0xffffe000u;
+  memcpy(&x, &u, 4);
+  return x;
+}
+
+int ref_sgemm_tf32(int terms, char transa, char transb, int64_t m, int64_t n, int64_t k, float alpha, const float* A,
+                   int64_t lda, const float* B, int64_t ldb, float beta, const float* C, int64_t ldc, float* Cout,
+                   double* S, int64_t ldo, const int64_t* cols, int64_t ncols) {
+  if (terms != 1 && terms != 3) return -1;
+  int bad = check_args(transa, transb, m, n, k, lda, ldb, ldc);
+  if (bad) return -bad - 1;
+  if (ldo < (m > 1 ? m : 1)) return -17;
+  if (m == 0 || n == 0) return 0;
+  const int ta = is_trans(transa), tb = is_trans(transb);
+  const int64_t nj = cols ? ncols : n;
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int64_t jj = 0; jj < nj; ++jj) {
+    const int64_t j = cols ? cols[jj] : jj;
+    for (int64_t i = 0; i < m; ++i) {
+      double acc = 0.0, mag = 0.0;
+      if (alpha != 0.0f) {
+        for (int64_t p = 0; p < k; ++p) {
+          const float a = ta ? A[p + i * lda] : A[i + p * lda];
+          const float b = tb ? B[j + p * ldb] : B[p + j * ldb];
+          const float ah = ref_tf32_round(a), bh = ref_tf32_round(b);
+          if (terms == 1) {
+            acc += (double)ah * (double)bh;
+          } else {
+            const float al = ref_tf32_round(a - ah), bl = ref_tf32_round(b - bh);
+            acc += (double)ah * (double)bh + (double)ah * (double)bl + (double)al * (double)bh;
+          }
+          mag += fabs((double)a) * fabs((double)b);
+        }
+      }
+      double r = (double)alpha * acc, s = fabs((double)alpha) * mag;
+      if (beta != 0.0f) {
+        r += (double)beta * (double)C[i + j * ldc];
+        s += fabs((double)beta) * fabs((double)C[i + j * ldc]);
+      }
+      Cout[i + j * ldo] = (float)r;
+      S[i + j * ldo] = s;
+    }
+  }
+  return 0;
+}
