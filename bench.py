@@ -178,6 +178,17 @@ def other_configs(b2, device):
             for tb in "NT":
                 real(kind, ta, tb, 1001, 999, 1003, 0.7, -0.3, "uniform", 4000, True,
                      f"{kind}gemm_{ta.lower()}{tb.lower()}_1001x999x1003_ld1027")
+    # fp32 on the tensor cores in TF32: reported separately, with the error each variant is specified with
+    for terms, err in ((1, "2^-10 * S"), (3, "fp32 level: (2^-21 + 2(3k+2) 2^-24) * S")):
+        for s in (4096, 8192):
+            A, lda, B, ldb, C, ldc = synth.gemm_inputs("N", "N", s, s, s, "uniform", 2100, torch.float32, device=device)
+            ws = torch.empty(b2.b2_sgemm_tf32_workspace_bytes(terms, s, s, s), dtype=torch.uint8, device=device)
+            g = quick_gflops(lambda: b2.b2_sgemm_tf32(terms, "N", "N", s, s, s, 1.5, A, lda, B, ldb, 0.5, C, ldc, ws),
+                             2.0 * s * s * s)
+            out.append({"workload": f"sgemm_tf32x{terms}_nn_{s}", "gflops": round(g, 1),
+                        "note": "tcgen05 kind::tf32, not FP32-FMA arithmetic; 2*m*n*k flops counted once; packing "
+                                "included", "error_bound_vs_fp32": err})
+            del A, B, C, ws
     m = n = k = 4096
     A = synth.matrix(m, k, m, "uniform", 5000, torch.complex128, device=device)
     B = synth.matrix(k, n, k, "uniform", 5002, torch.complex128, device=device)

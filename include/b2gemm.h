@@ -159,6 +159,27 @@ int b2_zgemm4m_static(char transa, char transb, int64_t m, int64_t n, int64_t k,
                       int64_t ldc, void* cuda_stream);
 
 /*
+ * fp32 GEMM on the tensor cores in TF32 -- separate entry points because TF32 changes results (b2_sgemm
+ * never uses it).  The paper has no counterpart; the operation is the same BLAS GEMM with the products taken
+ * in the TF32 format (1 sign, 8 exponent, 10 mantissa bits) and accumulated in fp32:
+ *   b2_sgemm_tf32x1   both operands rounded to nearest TF32 (ties away from zero): element error about
+ *                     2^-10 * (|alpha| |A||B|)_ij;
+ *   b2_sgemm_tf32x3   each operand split into a TF32 head and tail, the three leading products added
+ *                     (head*head + head*tail + tail*head): back at fp32 accuracy, three times the work.
+ * Same arguments, quick returns and error codes as b2_sgemm, plus a DEVICE workspace of at least
+ * b2_sgemm_tf32_workspace_bytes(terms, m, n, k) bytes (terms = 1 or 3), 256-byte aligned, owned by the caller
+ * and overwritten (it receives the packed, rounded K-major panels of op(A) and op(B)); argument 14.
+ * Any alignment and leading dimension of A, B, C is accepted.  Bounded device-side waits: b2_device_status.
+ */
+size_t b2_sgemm_tf32_workspace_bytes(int terms, int64_t m, int64_t n, int64_t k);
+int b2_sgemm_tf32x1(char transa, char transb, int64_t m, int64_t n, int64_t k, float alpha, const float* A,
+                    int64_t lda, const float* B, int64_t ldb, float beta, float* C, int64_t ldc, void* workspace,
+                    size_t workspace_bytes, void* cuda_stream);
+int b2_sgemm_tf32x3(char transa, char transb, int64_t m, int64_t n, int64_t k, float alpha, const float* A,
+                    int64_t lda, const float* B, int64_t ldb, float beta, float* C, int64_t ldc, void* workspace,
+                    size_t workspace_bytes, void* cuda_stream);
+
+/*
  * Host-buffer forms: A, B, C are HOST pointers (pinned memory makes the copies asynchronous),
  * dev_workspace is DEVICE memory of at least b2_gemm_host_workspace_bytes(...) bytes owned by
  * the caller.  The call copies the referenced parts of A and B (and C when beta != 0) to the

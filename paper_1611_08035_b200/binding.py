@@ -38,6 +38,9 @@ _SIGNATURES = {
                            c_void_p]),
     "b2_zgemm4m_static": (c_int, [c_char, c_char, c_int64, c_int64, c_int64, ctypes.POINTER(c_double), c_void_p, c_int64,
                                   c_void_p, c_int64, ctypes.POINTER(c_double), c_void_p, c_int64, c_void_p]),
+    "b2_sgemm_tf32_workspace_bytes": (c_size_t, [c_int, c_int64, c_int64, c_int64]),
+    "b2_sgemm_tf32x1": (c_int, _GEMM_TAIL_S + [c_void_p, c_size_t, c_void_p]),
+    "b2_sgemm_tf32x3": (c_int, _GEMM_TAIL_S + [c_void_p, c_size_t, c_void_p]),
     "b2_gemm_host_workspace_bytes": (c_size_t, [c_int, c_char, c_char, c_int64, c_int64, c_int64]),
     "b2_dgemm_host": (c_int, _GEMM_TAIL_D + [c_void_p, c_size_t, c_void_p]),
     "b2_sgemm_host": (c_int, _GEMM_TAIL_S + [c_void_p, c_size_t, c_void_p]),
@@ -253,3 +256,21 @@ def b2_device_status() -> int:
 def b2_selftest_wait_timeout() -> int:
     """Enqueue the bounded-wait self-test kernel (the next b2_device_status then reports B2_ERR_TIMEOUT)."""
     return lib().b2_selftest_wait_timeout(_stream())
+
+
+def b2_sgemm_tf32_workspace_bytes(terms: int, m: int, n: int, k: int) -> int:
+    return lib().b2_sgemm_tf32_workspace_bytes(terms, m, n, k)
+
+
+def b2_sgemm_tf32(terms, transa, transb, m, n, k, alpha, A, lda, B, ldb, beta, C, ldc, workspace, check=True) -> int:
+    """fp32 GEMM on the tensor cores in TF32 (terms=1: b2_sgemm_tf32x1, terms=3: b2_sgemm_tf32x3); device tensors."""
+    for t in (A, B, C):
+        if t is not None and (t.dtype != torch.float32 or not t.is_cuda):
+            raise TypeError("b2_sgemm_tf32 takes float32 CUDA tensors")
+    fn = {1: lib().b2_sgemm_tf32x1, 3: lib().b2_sgemm_tf32x3}[terms]
+    wbytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    rc = fn(_tr(transa), _tr(transb), m, n, k, alpha, _ptr(A), lda, _ptr(B), ldb, beta, _ptr(C), ldc, _ptr(workspace),
+            wbytes, _stream())
+    if check:
+        _check(f"b2_sgemm_tf32x{terms}", rc)
+    return rc

@@ -7,6 +7,7 @@
 #include "gemm_tma.cuh"
 
 namespace b2 {
+int tf32_take_status();  // status word of the TF32 tensor-core kernels (sgemm_tf32.cu)
 namespace {
 
 // Status word the TMA kernels write when a bounded wait runs out; read and cleared by b2_device_status.
@@ -150,5 +151,6 @@ extern "C" int b2_device_status(void* cuda_stream) {
     const int zero = 0;
     if (cudaMemcpyToSymbol(b2::g_device_status, &zero, sizeof(int)) != cudaSuccess) return B2_ERR_LAUNCH;
   }
-  return value;
+  const int other = b2::tf32_take_status();
+  return value != 0 ? value : other;
 }
