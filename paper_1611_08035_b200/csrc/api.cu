@@ -164,6 +164,9 @@ int gemm_entry(int variant, char transa, char transb, int64_t m, int64_t n, int6
   const VariantInfo& vi = variant_info_t<T>(variant);
   const double resident = (double)sm_count_cached() * vi.ctas_per_sm;
   int group_m = (int)(sqrt(resident * vi.bn / vi.bm) + 0.5);
+  // Measured at 8192^3 (DRAM bytes of one launch): 12 tile rows per group read the least for every tile shape
+  // (64x64: 13.2 GB against 15.8 GB at 24 rows and 64 GB without grouping; 128x128: 7.6 GB), at unchanged speed.
+  if (group_m > 12) group_m = 12;
   args.group_m = group_m < 1 ? 1 : group_m;
   return variant_launch_t<T>(variant)(args, is_t(transa), is_t(transb), operands_aligned(A, lda, B, ldb), stream);
 }
