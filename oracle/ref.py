@@ -46,6 +46,9 @@ def lib() -> ctypes.CDLL:
                                                               c_void_p, c_int64, c_void_p, c_void_p, c_int64, c_void_p,
                                                               c_int64]
         _lib.ref_sgemm_tf32.restype = c_int
+        _lib.ref_dsyrk.argtypes = [c_char, c_char, c_int64, c_int64, c_double, c_void_p, c_int64, c_double, c_void_p, c_int64]
+        _lib.ref_ssyrk.argtypes = [c_char, c_char, c_int64, c_int64, c_float, c_void_p, c_int64, c_float, c_void_p, c_int64]
+        _lib.ref_dsyrk.restype = _lib.ref_ssyrk.restype = c_int
         for fn in ("ref_dgemm", "ref_sgemm", "ref_dgemm_hi", "ref_sgemm_hi", "ref_zgemm", "ref_zgemm_hi",
                    "ref_num_threads"):
             getattr(_lib, fn).restype = c_int
@@ -207,3 +210,31 @@ def ref_sgemm_tf32(terms, transa, transb, m, n, k, alpha, A, lda, B, ldb, beta, 
         raise ValueError(f"oracle rejected argument {-rc}")
     del keep
     return out, S
+
+
+def ref_syrk(uplo, trans, n, k, alpha, A, lda, beta, C, ldc) -> None:
+    """C := alpha*A*A^T + beta*C (trans N) or alpha*A^T*A + beta*C (trans T) on the uplo triangle of C, in place."""
+    dt = C.dtype
+    _flat(A, dt), _flat(C, dt)
+    if dt == np.float64:
+        fn, a, b = lib().ref_dsyrk, float(alpha), float(beta)
+    elif dt == np.float32:
+        fn, a, b = lib().ref_ssyrk, float(np.float32(alpha)), float(np.float32(beta))
+    else:
+        raise TypeError(f"unsupported dtype {dt}")
+    if n > 0:
+        _need(C, ldc, n, n, "C")
+        if alpha != 0 and k > 0:
+            tr = trans in "TtCc"
+            _need(A, lda, n if tr else k, k if tr else n, "A")
+    rc = fn(_tr(uplo), _tr(trans), n, k, a, A.ctypes.data, lda, b, C.ctypes.data, ldc)
+    if rc != 0:
+        raise ValueError(f"oracle rejected argument {-rc}")
+
+
+def ref_gemm_strided_batched(transa, transb, m, n, k, alpha, A, lda, stride_a, B, ldb, stride_b, beta, C, ldc,
+                             stride_c, batch) -> None:
+    """`batch` independent GEMMs on operands that start stride_* elements apart: one ref_gemm call per problem."""
+    for b in range(batch):
+        ref_gemm(transa, transb, m, n, k, alpha, A[b * stride_a:], lda, B[b * stride_b:], ldb, beta,
+                 C[b * stride_c:], ldc)

@@ -298,3 +298,57 @@ int ref_sgemm_tf32(int terms, char transa, char transb, int64_t m, int64_t n, in
   }
   return 0;
 }
+
+/*
+ * Symmetric rank-k update, the level-3 routine that is a GEMM restricted to one triangle (the paper names the
+ * level-3 BLAS as consumers of the GEMM kernel, Abstract and Introduction; the definition is the BLAS one):
+ *     trans = N:  C := alpha * A * A^T + beta * C,   A is n x k
+ *     trans = T:  C := alpha * A^T * A + beta * C,   A is k x n
+ * Only the triangle named by uplo ('L': i >= j, 'U': i <= j) of the n x n matrix C is read or written.
+ * Same arithmetic rules as ref_*gemm: ascending p, one multiply and one add per term, beta == 0 does not read C,
+ * alpha == 0 or k == 0 scales the triangle only.
+ */
+#define DEFINE_REF_SYRK(NAME, T)                                                                          \
+  int NAME(char uplo, char trans, int64_t n, int64_t k, T alpha, const T* A, int64_t lda, T beta, T* C,   \
+           int64_t ldc) {                                                                                  \
+    const int lower = (uplo == 'L' || uplo == 'l'), upper = (uplo == 'U' || uplo == 'u');                  \
+    if (!lower && !upper) return -1;                                                                       \
+    if (!is_trans(trans) && !is_notrans(trans)) return -2;                                                 \
+    if (n < 0) return -3;                                                                                  \
+    if (k < 0) return -4;                                                                                  \
+    const int tr = is_trans(trans);                                                                        \
+    const int64_t rows_a = tr ? k : n;                                                                     \
+    if (lda < (rows_a > 1 ? rows_a : 1)) return -7;                                                        \
+    if (ldc < (n > 1 ? n : 1)) return -10;                                                                 \
+    if (n == 0) return 0;                                                                                  \
+    const int scale_only = (alpha == (T)0 || k == 0);                                                      \
+    if (scale_only && beta == (T)1) return 0;                                                              \
+    _Pragma("omp parallel for schedule(dynamic, 1)") for (int64_t j = 0; j < n; ++j) {                     \
+      const int64_t i_lo = lower ? j : 0, i_hi = lower ? n : j + 1;                                        \
+      for (int64_t i = i_lo; i < i_hi; ++i) {                                                              \
+        T acc = (T)0;                                                                                      \
+        if (!scale_only) {                                                                                 \
+          for (int64_t p = 0; p < k; ++p) {                                                                \
+            const T a = tr ? A[p + i * lda] : A[i + p * lda];                                              \
+            const T b = tr ? A[p + j * lda] : A[j + p * lda];                                              \
+            const T prod = a * b;                                                                          \
+            acc = acc + prod;                                                                              \
+          }                                                                                                \
+        }                                                                                                  \
+        T* c = &C[i + j * ldc];                                                                            \
+        if (scale_only) {                                                                                  \
+          *c = (beta == (T)0) ? (T)0 : beta * *c;                                                          \
+        } else if (beta == (T)0) {                                                                         \
+          *c = alpha * acc;                                                                                \
+        } else {                                                                                           \
+          const T t1 = alpha * acc;                                                                        \
+          const T t2 = beta * *c;                                                                          \
+          *c = t1 + t2;                                                                                    \
+        }                                                                                                  \
+      }                                                                                                    \
+    }                                                                                                      \
+    return 0;                                                                                              \
+  }
+
+DEFINE_REF_SYRK(ref_dsyrk, double)
+DEFINE_REF_SYRK(ref_ssyrk, float)
