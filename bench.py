@@ -179,6 +179,23 @@ def other_configs(b2, device):
             for tb in "NT":
                 real(kind, ta, tb, 1001, 999, 1003, 0.7, -0.3, "uniform", 4000, True,
                      f"{kind}gemm_{ta.lower()}{tb.lower()}_1001x999x1003_ld1027")
+    # level-3 consumers of the kernel: symmetric rank-k update (n*n*k flops: half of the GEMM) and a strided batch
+    for n_, k_ in ((8192, 8192), (16384, 256)):
+        A = synth.matrix(n_, k_, n_, "uniform", 7000, torch.float64, device=device)
+        C = synth.matrix(n_, n_, n_, "uniform", 7001, torch.float64, device=device)
+        g = quick_gflops(lambda: b2.b2_syrk("L", "N", n_, k_, -1.0, A, n_, 1.0, C, n_), 1.0 * n_ * n_ * k_)
+        out.append({"workload": f"dsyrk_ln_n{n_}_k{k_}", "gflops": round(g, 1), "frac_of_peak": round(g / 1e3 / FP64_PEAK_TFLOPS, 4),
+                    "note": "n*n*k flops (stored triangle only)"})
+        del A, C
+    bm, bb = 512, 64
+    A = synth.matrix(bm, bm * bb, bm, "uniform", 7100, torch.float64, device=device)
+    B = synth.matrix(bm, bm * bb, bm, "uniform", 7101, torch.float64, device=device)
+    C = synth.matrix(bm, bm * bb, bm, "uniform", 7102, torch.float64, device=device)
+    g = quick_gflops(lambda: b2.b2_gemm_strided_batched("N", "N", bm, bm, bm, 1.5, A, bm, bm * bm, B, bm, bm * bm, 0.5, C,
+                                                        bm, bm * bm, bb), 2.0 * bm ** 3 * bb)
+    out.append({"workload": f"dgemm_strided_batched_{bb}x{bm}^3", "gflops": round(g, 1),
+                "frac_of_peak": round(g / 1e3 / FP64_PEAK_TFLOPS, 4)})
+    del A, B, C
     # fp32 on the tensor cores in TF32: reported separately, with the error each variant is specified with
     for terms, err in ((1, "2^-10 * S"), (3, "fp32 level: (2^-21 + 2(3k+2) 2^-24) * S")):
         for s in (4096, 8192):

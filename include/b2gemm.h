@@ -159,6 +159,35 @@ int b2_zgemm4m_static(char transa, char transb, int64_t m, int64_t n, int64_t k,
                       int64_t ldc, void* cuda_stream);
 
 /*
+ * Symmetric rank-k update on the GEMM kernel (the paper names the level-3 BLAS as consumers of its kernel,
+ * Abstract and Introduction; the definition is the BLAS one):
+ *     trans = N:  C := alpha*A*A^T + beta*C,  A is n x k;      trans = T (or C):  C := alpha*A^T*A + beta*C,  A is k x n.
+ * Only the triangle of the n x n matrix C named by uplo ('L': i >= j, 'U': i <= j) is read or written; tiles of
+ * the other triangle are not computed.  Device pointers, column-major, conventions as b2_dgemm.  Argument
+ * numbering for -i: uplo 1, trans 2, n 3, k 4, alpha 5, A 6, lda 7, beta 8, C 9, ldc 10.
+ * lda >= max(1, trans==N ? n : k), ldc >= max(1, n).  alpha == 0 or k == 0 scales the triangle by beta.
+ */
+int b2_dsyrk(char uplo, char trans, int64_t n, int64_t k, double alpha, const double* A, int64_t lda, double beta,
+             double* C, int64_t ldc, void* cuda_stream);
+int b2_ssyrk(char uplo, char trans, int64_t n, int64_t k, float alpha, const float* A, int64_t lda, float beta,
+             float* C, int64_t ldc, void* cuda_stream);
+
+/*
+ * Strided-batched GEMM: `batch` independent problems C_b := alpha*op(A_b)*op(B_b) + beta*C_b of one shape, where
+ * A_b = A + b*stride_a, B_b = B + b*stride_b, C_b = C + b*stride_c (strides in elements; stride_a / stride_b may
+ * be 0 to share an operand; for batch > 1 stride_c must be at least ldc*(n-1) + m so that results do not overlap).
+ * One launch covers up to 65535 problems (the batch index is the grid's second dimension).  Conventions as
+ * b2_dgemm.  Argument numbering for -i: transa 1, transb 2, m 3, n 4, k 5, alpha 6, A 7, lda 8, stride_a 9, B 10,
+ * ldb 11, stride_b 12, beta 13, C 14, ldc 15, stride_c 16, batch 17.
+ */
+int b2_dgemm_strided_batched(char transa, char transb, int64_t m, int64_t n, int64_t k, double alpha, const double* A,
+                             int64_t lda, int64_t stride_a, const double* B, int64_t ldb, int64_t stride_b,
+                             double beta, double* C, int64_t ldc, int64_t stride_c, int64_t batch, void* cuda_stream);
+int b2_sgemm_strided_batched(char transa, char transb, int64_t m, int64_t n, int64_t k, float alpha, const float* A,
+                             int64_t lda, int64_t stride_a, const float* B, int64_t ldb, int64_t stride_b, float beta,
+                             float* C, int64_t ldc, int64_t stride_c, int64_t batch, void* cuda_stream);
+
+/*
  * fp32 GEMM on the tensor cores in TF32 -- separate entry points because TF32 changes results (b2_sgemm
  * never uses it).  The paper has no counterpart; the operation is the same BLAS GEMM with the products taken
  * in the TF32 format (1 sign, 8 exponent, 10 mantissa bits) and accumulated in fp32:

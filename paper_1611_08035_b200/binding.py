@@ -38,6 +38,16 @@ _SIGNATURES = {
                            c_void_p]),
     "b2_zgemm4m_static": (c_int, [c_char, c_char, c_int64, c_int64, c_int64, ctypes.POINTER(c_double), c_void_p, c_int64,
                                   c_void_p, c_int64, ctypes.POINTER(c_double), c_void_p, c_int64, c_void_p]),
+    "b2_dsyrk": (c_int, [c_char, c_char, c_int64, c_int64, c_double, c_void_p, c_int64, c_double, c_void_p, c_int64,
+                         c_void_p]),
+    "b2_ssyrk": (c_int, [c_char, c_char, c_int64, c_int64, c_float, c_void_p, c_int64, c_float, c_void_p, c_int64,
+                         c_void_p]),
+    "b2_dgemm_strided_batched": (c_int, [c_char, c_char, c_int64, c_int64, c_int64, c_double, c_void_p, c_int64, c_int64,
+                                         c_void_p, c_int64, c_int64, c_double, c_void_p, c_int64, c_int64, c_int64,
+                                         c_void_p]),
+    "b2_sgemm_strided_batched": (c_int, [c_char, c_char, c_int64, c_int64, c_int64, c_float, c_void_p, c_int64, c_int64,
+                                         c_void_p, c_int64, c_int64, c_float, c_void_p, c_int64, c_int64, c_int64,
+                                         c_void_p]),
     "b2_sgemm_tf32_workspace_bytes": (c_size_t, [c_int, c_int64, c_int64, c_int64]),
     "b2_sgemm_tf32x1": (c_int, _GEMM_TAIL_S + [c_void_p, c_size_t, c_void_p]),
     "b2_sgemm_tf32x3": (c_int, _GEMM_TAIL_S + [c_void_p, c_size_t, c_void_p]),
@@ -273,4 +283,36 @@ def b2_sgemm_tf32(terms, transa, transb, m, n, k, alpha, A, lda, B, ldb, beta, C
             wbytes, _stream())
     if check:
         _check(f"b2_sgemm_tf32x{terms}", rc)
+    return rc
+
+
+def b2_syrk(uplo, trans, n, k, alpha, A, lda, beta, C, ldc, check=True) -> int:
+    """Symmetric rank-k update on the uplo triangle of C (b2_dsyrk / b2_ssyrk by dtype); device tensors."""
+    if C is not None and C.dtype == torch.float32:
+        fn, name = lib().b2_ssyrk, "b2_ssyrk"
+    else:
+        fn, name = lib().b2_dsyrk, "b2_dsyrk"
+    for t in (A, C):
+        if t is not None and (not t.is_cuda or (C is not None and t.dtype != C.dtype)):
+            raise TypeError(f"{name} takes CUDA tensors of one dtype")
+    rc = fn(_tr(uplo), _tr(trans), n, k, alpha, _ptr(A), lda, beta, _ptr(C), ldc, _stream())
+    if check:
+        _check(name, rc)
+    return rc
+
+
+def b2_gemm_strided_batched(transa, transb, m, n, k, alpha, A, lda, stride_a, B, ldb, stride_b, beta, C, ldc, stride_c,
+                            batch, check=True) -> int:
+    """`batch` GEMMs of one shape on strided operands (b2_dgemm_strided_batched / b2_sgemm_strided_batched)."""
+    if C is not None and C.dtype == torch.float32:
+        fn, name = lib().b2_sgemm_strided_batched, "b2_sgemm_strided_batched"
+    else:
+        fn, name = lib().b2_dgemm_strided_batched, "b2_dgemm_strided_batched"
+    for t in (A, B, C):
+        if t is not None and (not t.is_cuda or (C is not None and t.dtype != C.dtype)):
+            raise TypeError(f"{name} takes CUDA tensors of one dtype")
+    rc = fn(_tr(transa), _tr(transb), m, n, k, alpha, _ptr(A), lda, stride_a, _ptr(B), ldb, stride_b, beta, _ptr(C), ldc,
+            stride_c, batch, _stream())
+    if check:
+        _check(name, rc)
     return rc

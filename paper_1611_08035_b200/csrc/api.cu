@@ -45,7 +45,7 @@ const LaunchFn<double> kF64Launch[] = {launch_f64_v0, launch_f64_v1, launch_f64_
 const VariantInfo kF32Info[] = {
     {"ffma2_128x128x16_s4", "ffma2", 128, 128, 16, 4, 256, 2, 0.72},
     {"ffma2_128x64x16_s4", "ffma2", 128, 64, 16, 4, 128, 3, 0.775},
-    {"ffma2_64x64x16_s4", "ffma2", 64, 64, 16, 4, 64, 8, 0.68},
+    {"ffma2_64x64x16_s4", "ffma2", 64, 64, 16, 4, 64, 6, 0.68},
     {"ffma_128x64x16_s4", "ffma", 128, 64, 16, 4, 128, 4, 0.70},
 };
 const LaunchFn<float> kF32Launch[] = {launch_f32_v0, launch_f32_v1, launch_f32_v2, launch_f32_v3};
@@ -134,6 +134,41 @@ int choose_variant(int64_t m, int64_t n, int64_t k, bool aligned) {
   return select_tile(cand, count < 16 ? count : 16, m, n, k, sm_count_cached(), (int)sizeof(T));
 }
 
+// Variant choice and launch of an already checked, non-trivial problem (m, n, k > 0, alpha != 0).
+template <typename T>
+int gemm_launch_checked(int variant, bool ta, bool tb, int64_t m, int64_t n, int64_t k, T alpha, const T* A,
+                        int64_t lda, const T* B, int64_t ldb, T beta, T* C, int64_t ldc, const GemmExtra& ex,
+                        cudaStream_t stream) {
+  // TMA staging needs 16-byte aligned columns and one tensor map per operand, so it serves single problems only
+  // (every problem of a batch must start on a 16-byte boundary for the 16-byte staging path)
+  constexpr int64_t kVec = 16 / (int64_t)sizeof(T);
+  const bool aligned = operands_aligned(A, lda, B, ldb) &&
+                       (ex.batch <= 1 || (ex.stride_a % kVec == 0 && ex.stride_b % kVec == 0));
+  if (variant == B2_VARIANT_AUTO) variant = choose_variant<T>(m, n, k, aligned && ex.batch <= 1);
+  GemmArgs<T> args;
+  args.m = m, args.n = n, args.k = k;
+  args.alpha = alpha, args.beta = beta;
+  args.A = A, args.lda = lda, args.B = B, args.ldb = ldb, args.C = C, args.ldc = ldc;
+  args.tiles_m = args.tiles_n = 0;
+  args.tri = ex.tri;
+  args.batch = ex.batch, args.batch_a = ex.stride_a, args.batch_b = ex.stride_b, args.batch_c = ex.stride_c;
+  // Rasterisation group: the CTAs resident at one time should cover a block of C whose A row-panels and
+  // B column-panels have about the same size: group_m * BM = (resident / group_m) * BN.
+  const VariantInfo& vi = variant_info_t<T>(variant);
+  const double resident = (double)sm_count_cached() * vi.ctas_per_sm;
+  int group_m = (int)(sqrt(resident * vi.bn / vi.bm) + 0.5);
+  // Measured at 8192^3 (DRAM bytes of one launch): 12 tile rows per group read the least for every tile shape
+  // (64x64: 13.2 GB against 15.8 GB at 24 rows and 64 GB without grouping; 128x128: 7.6 GB), at unchanged speed.
+  if (group_m > 12) group_m = 12;
+  args.group_m = group_m < 1 ? 1 : group_m;
+  return variant_launch_t<T>(variant)(args, ta, tb, aligned, stream);
+}
+template int gemm_launch_checked<double>(int, bool, bool, int64_t, int64_t, int64_t, double, const double*, int64_t,
+                                         const double*, int64_t, double, double*, int64_t, const GemmExtra&,
+                                         cudaStream_t);
+template int gemm_launch_checked<float>(int, bool, bool, int64_t, int64_t, int64_t, float, const float*, int64_t,
+                                        const float*, int64_t, float, float*, int64_t, const GemmExtra&, cudaStream_t);
+
 template <typename T>
 int gemm_entry(int variant, char transa, char transb, int64_t m, int64_t n, int64_t k, T alpha, const T* A,
                int64_t lda, const T* B, int64_t ldb, T beta, T* C, int64_t ldc, void* cuda_stream) {
@@ -153,22 +188,8 @@ int gemm_entry(int variant, char transa, char transb, int64_t m, int64_t n, int6
     scale_kernel<T><<<(unsigned)blocks, threads, 0, stream>>>(m, n, beta, C, ldc);
     return cudaGetLastError() == cudaSuccess ? B2_OK : B2_ERR_LAUNCH;
   }
-  if (variant == B2_VARIANT_AUTO) variant = choose_variant<T>(m, n, k, operands_aligned(A, lda, B, ldb));
-  GemmArgs<T> args;
-  args.m = m, args.n = n, args.k = k;
-  args.alpha = alpha, args.beta = beta;
-  args.A = A, args.lda = lda, args.B = B, args.ldb = ldb, args.C = C, args.ldc = ldc;
-  args.tiles_m = args.tiles_n = 0;
-  // Rasterisation group: the CTAs resident at one time should cover a block of C whose A row-panels and
-  // B column-panels have about the same size: group_m * BM = (resident / group_m) * BN.
-  const VariantInfo& vi = variant_info_t<T>(variant);
-  const double resident = (double)sm_count_cached() * vi.ctas_per_sm;
-  int group_m = (int)(sqrt(resident * vi.bn / vi.bm) + 0.5);
-  // Measured at 8192^3 (DRAM bytes of one launch): 12 tile rows per group read the least for every tile shape
-  // (64x64: 13.2 GB against 15.8 GB at 24 rows and 64 GB without grouping; 128x128: 7.6 GB), at unchanged speed.
-  if (group_m > 12) group_m = 12;
-  args.group_m = group_m < 1 ? 1 : group_m;
-  return variant_launch_t<T>(variant)(args, is_t(transa), is_t(transb), operands_aligned(A, lda, B, ldb), stream);
+  return gemm_launch_checked<T>(variant, is_t(transa), is_t(transb), m, n, k, alpha, A, lda, B, ldb, beta, C, ldc,
+                                GemmExtra(), stream);
 }
 
 // Explicit instantiations used by the other translation units (complex and host-buffer entries).

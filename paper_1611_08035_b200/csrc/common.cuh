@@ -19,7 +19,22 @@ struct GemmArgs {
   int64_t ldc;
   int tiles_m, tiles_n;  // CTA-tile counts along m and n
   int group_m;           // rasterisation: tile rows per group
+  int tri;               // 0: all of C;  1: only i >= j (lower triangle);  2: only i <= j (upper triangle)
+  int batch;             // number of problems of a strided batch (grid.y), at most 65535 per launch
+  int64_t batch_a, batch_b, batch_c;  // element offsets between the operands of consecutive problems
 };
+
+// Does the BM x BN tile at (m0, n0) lie entirely outside the stored triangle?
+__device__ __forceinline__ bool tile_outside_triangle(int tri, int64_t m0, int64_t n0, int bm, int bn) {
+  return (tri == 1 && n0 > m0 + bm - 1) || (tri == 2 && m0 > n0 + bn - 1);
+}
+// Does it cross the diagonal (so that single elements have to be masked)?
+__device__ __forceinline__ bool tile_crosses_diagonal(int tri, int64_t m0, int64_t n0, int bm, int bn) {
+  return tri != 0 && !((tri == 1 && m0 >= n0 + bn - 1) || (tri == 2 && n0 >= m0 + bm - 1));
+}
+__device__ __forceinline__ bool in_triangle(int tri, int64_t row, int64_t col) {
+  return tri == 0 || (tri == 1 ? row >= col : row <= col);
+}
 
 // ---- cp.async (global -> shared, asynchronous, zero-filling past src_bytes) -------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {

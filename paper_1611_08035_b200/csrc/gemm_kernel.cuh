@@ -58,30 +58,32 @@ struct Stager {
   static constexpr int Q = STRAIGHT ? 1 : BO / LSTEP;           // transposing: passes that cover the o-extent once
   static_assert(STRAIGHT || (NT % RUN == 0 && BO % LSTEP == 0 && BK % RUN == 0), "transposing copy geometry");
 
-  const T* src;    // this thread's first chunk of the next slab to stage
-  int64_t lstep;   // source elements between the lines of consecutive passes
-  int64_t kstep;   // source elements to advance by one slab (BK along k)
-  int dst0;        // element offset of this thread's first chunk inside a stage
+  const T* src;  // this thread's first chunk of the next slab to stage (the only per-thread state)
 
-  __device__ __forceinline__ void init(const T* X0, int64_t ld, int tid) {
-    lstep = (int64_t)LSTEP * ld;
+  // element offset of the thread's first chunk inside a stage
+  static __device__ __forceinline__ int dst0_of(int tid) {
     if constexpr (STRAIGHT) {
-      const int line = tid / CPL, cc = (tid % CPL) * VEC;
-      src = X0 + cc + (int64_t)line * ld;
-      dst0 = line * PITCH + cc;
-      kstep = (SRC == OC) ? (int64_t)BK * ld : (int64_t)BK;
+      return (tid / CPL) * PITCH + (tid % CPL) * VEC;
     } else {
-      const int kk = tid % RUN, o = tid / RUN;
-      src = X0 + kk + (int64_t)o * ld;
-      dst0 = kk * PITCH + o;
-      kstep = BK;
+      return (tid % RUN) * PITCH + tid / RUN;
     }
   }
 
-  __device__ __forceinline__ void advance() { src += kstep; }
+  __device__ __forceinline__ void init(const T* X0, int64_t ld, int tid) {
+    if constexpr (STRAIGHT) {
+      src = X0 + (tid % CPL) * VEC + (int64_t)(tid / CPL) * ld;
+    } else {
+      src = X0 + (tid % RUN) + (int64_t)(tid / RUN) * ld;
+    }
+  }
+
+  // advance by one slab (BK along k)
+  __device__ __forceinline__ void advance(int64_t ld) { src += (STRAIGHT && SRC == OC) ? (int64_t)BK * ld : (int64_t)BK; }
 
   // Slab fully inside the operand: no predicates.
-  __device__ __forceinline__ void load_fast(T* __restrict__ s) const {
+  __device__ __forceinline__ void load_fast(T* __restrict__ s, int64_t ld, int tid) const {
+    const int64_t lstep = (int64_t)LSTEP * ld;  // source elements between the lines of consecutive passes
+    const int dst0 = dst0_of(tid);
 #pragma unroll
     for (int it = 0; it < ITER; ++it) {
       if constexpr (STRAIGHT) {
@@ -97,7 +99,9 @@ struct Stager {
   // are skipped, not zero-filled: whatever the shared-memory rows beyond o_valid hold only feeds accumulators of
   // rows/columns >= m or n of C, which the epilogue never stores.  A chunk that straddles the edge copies its
   // valid bytes only.  No address outside the operand is formed into a load.
-  __device__ __forceinline__ void load_edge(T* __restrict__ s, int o_valid, int tid) const {
+  __device__ __forceinline__ void load_edge(T* __restrict__ s, int64_t ld, int o_valid, int tid) const {
+    const int64_t lstep = (int64_t)LSTEP * ld;
+    const int dst0 = dst0_of(tid);
 #pragma unroll
     for (int it = 0; it < ITER; ++it) {
       if constexpr (STRAIGHT) {
@@ -240,17 +244,20 @@ struct DmmaMicro {
   // The old C values are fetched in batches, all loads of a batch issued before the first
   // store, so their latencies overlap instead of adding up (a store to C may alias a later
   // load of C as far as the compiler can tell).
-  static __device__ __forceinline__ void epilogue(const Acc& acc, const GemmArgs<double>& p, int64_t m0, int64_t n0,
-                                                  int warp_m, int warp_n, int lane) {
+  static __device__ __forceinline__ void epilogue(const Acc& acc, const GemmArgs<double>& p, double* C, int64_t m0,
+                                                  int64_t n0, int warp_m, int warp_n, int lane) {
     const int g = lane >> 2, t = lane & 3;
-    const bool vec_ok = ((reinterpret_cast<uintptr_t>(p.C) & 15) == 0) && ((p.ldc & 1) == 0);
+    const bool vec_ok = ((reinterpret_cast<uintptr_t>(C) & 15) == 0) && ((p.ldc & 1) == 0);
     const bool use_beta = (p.beta != 0.0);
     // old values in flight per batch: 32 doubles when the register budget is 255, 16 when it is 128
     constexpr int BATCH = (MI * NI * 4 >= 64) ? 32 : 16;
     constexpr int NB = (BATCH / (MI * 4)) > 0 ? ((BATCH / (MI * 4)) < NI ? (BATCH / (MI * 4)) : NI) : 1;
     static_assert(NI % NB == 0, "batches must tile the fragment columns");
+    // this lane's first element, and how many rows / columns of C remain from there (32-bit from here on)
     const int64_t row0 = m0 + warp_m * WTM + 2 * g;
     const int64_t col0 = n0 + warp_n * WTN + 2 * t;
+    double* base = C + col0 * p.ldc + row0;
+    const int rows_left = (int)min((int64_t)BM, p.m - row0), cols_left = (int)min((int64_t)BN, p.n - col0);
 #pragma unroll
     for (int nb0 = 0; nb0 < NI; nb0 += NB) {
       double2 old[NB][2][MI];
@@ -261,15 +268,15 @@ struct DmmaMicro {
           for (int h = 0; h < 2; ++h)
 #pragma unroll
             for (int mi = 0; mi < MI; ++mi) {
-              const int64_t col = col0 + (nb0 + nb) * 8 + h, row = row0 + mi * 16;
+              const int col = (nb0 + nb) * 8 + h, row = mi * 16;
               old[nb][h][mi] = make_double2(0.0, 0.0);
-              if (col < p.n && row < p.m) {
-                const double* src = p.C + col * p.ldc + row;
-                if (vec_ok && row + 1 < p.m) {
+              if (col < cols_left && row < rows_left) {
+                const double* src = base + col * p.ldc + row;
+                if (vec_ok && row + 1 < rows_left) {
                   old[nb][h][mi] = *reinterpret_cast<const double2*>(src);
                 } else {
                   old[nb][h][mi].x = src[0];
-                  if (row + 1 < p.m) old[nb][h][mi].y = src[1];
+                  if (row + 1 < rows_left) old[nb][h][mi].y = src[1];
                 }
               }
             }
@@ -280,22 +287,45 @@ struct DmmaMicro {
         for (int h = 0; h < 2; ++h)
 #pragma unroll
           for (int mi = 0; mi < MI; ++mi) {
-            const int64_t col = col0 + (nb0 + nb) * 8 + h, row = row0 + mi * 16;
-            if (col >= p.n || row >= p.m) continue;
+            const int col = (nb0 + nb) * 8 + h, row = mi * 16;
+            if (col >= cols_left || row >= rows_left) continue;
             double v0 = p.alpha * acc.c[mi][nb0 + nb][h], v1 = p.alpha * acc.c[mi][nb0 + nb][2 + h];
             if (use_beta) {
               v0 += p.beta * old[nb][h][mi].x;
               v1 += p.beta * old[nb][h][mi].y;
             }
-            double* dst = p.C + col * p.ldc + row;
-            if (vec_ok && row + 1 < p.m) {
+            double* dst = base + col * p.ldc + row;
+            if (vec_ok && row + 1 < rows_left) {
               *reinterpret_cast<double2*>(dst) = make_double2(v0, v1);
             } else {
               dst[0] = v0;
-              if (row + 1 < p.m) dst[1] = v1;
+              if (row + 1 < rows_left) dst[1] = v1;
             }
           }
     }
+  }
+
+  // Element-wise epilogue for tiles that cross the diagonal of a triangular update: only elements inside the
+  // stored triangle are read or written.
+  static __device__ __forceinline__ void epilogue_masked(const Acc& acc, const GemmArgs<double>& p, double* C,
+                                                         int64_t m0, int64_t n0, int warp_m, int warp_n, int lane) {
+    const int g = lane >> 2, t = lane & 3;
+    const bool use_beta = (p.beta != 0.0);
+#pragma unroll
+    for (int mi = 0; mi < MI; ++mi)
+#pragma unroll
+      for (int ni = 0; ni < NI; ++ni)
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+          const int64_t row = m0 + warp_m * WTM + mi * 16 + 2 * g + (r >> 1);
+          const int64_t col = n0 + warp_n * WTN + ni * 8 + 2 * t + (r & 1);
+          if (row < p.m && col < p.n && in_triangle(p.tri, row, col)) {
+            double* dst = C + col * p.ldc + row;
+            double v = p.alpha * acc.c[mi][ni][r];
+            if (use_beta) v += p.beta * *dst;
+            *dst = v;
+          }
+        }
   }
 };
 
@@ -417,10 +447,10 @@ struct SimtMicro {
   }
 
   // C := alpha*acc + beta*C; old C values are fetched in batches of columns before any store of the batch.
-  static __device__ __forceinline__ void epilogue(const Acc& acc, const GemmArgs<T>& p, int64_t m0, int64_t n0,
+  static __device__ __forceinline__ void epilogue(const Acc& acc, const GemmArgs<T>& p, T* C, int64_t m0, int64_t n0,
                                                   int warp_m, int warp_n, int lane) {
     const int lx = lane & 7, ly = lane >> 3;
-    const bool vec_ok = ((reinterpret_cast<uintptr_t>(p.C) & 15) == 0) && ((p.ldc % VEC) == 0);
+    const bool vec_ok = ((reinterpret_cast<uintptr_t>(C) & 15) == 0) && ((p.ldc % VEC) == 0);
     const bool use_beta = (p.beta != T(0));
     constexpr int JB = 2;  // columns per batch: 16 old values in flight
     const int64_t row0 = m0 + warp_m * WTM + lx * VEC;
@@ -439,7 +469,7 @@ struct SimtMicro {
 #pragma unroll
             for (int e = 0; e < VEC; ++e) old[jb][gi * VEC + e] = T(0);
             if (col < p.n && row < p.m) {
-              const T* src = p.C + col * p.ldc + row;
+              const T* src = C + col * p.ldc + row;
               if (vec_ok && row + VEC <= p.m) {
                 load_vec(&old[jb][gi * VEC], src);
               } else {
@@ -466,7 +496,7 @@ struct SimtMicro {
             v[e] = p.alpha * get(acc, gi * VEC + e, j);
             if (use_beta) v[e] += p.beta * old[jb][gi * VEC + e];
           }
-          T* dst = p.C + col * p.ldc + row;
+          T* dst = C + col * p.ldc + row;
           if (vec_ok && row + VEC <= p.m) {
             VT out;
             if constexpr (sizeof(T) == 4) {
@@ -480,6 +510,26 @@ struct SimtMicro {
             for (int e = 0; e < VEC; ++e)
               if (row + e < p.m) dst[e] = v[e];
           }
+        }
+      }
+    }
+  }
+  // Element-wise epilogue for tiles that cross the diagonal of a triangular update.
+  static __device__ __forceinline__ void epilogue_masked(const Acc& acc, const GemmArgs<T>& p, T* C, int64_t m0,
+                                                         int64_t n0, int warp_m, int warp_n, int lane) {
+    const int lx = lane & 7, ly = lane >> 3;
+    const bool use_beta = (p.beta != T(0));
+#pragma unroll
+    for (int j = 0; j < TN; ++j) {
+      const int64_t col = n0 + warp_n * WTN + (j / VEC) * 4 * VEC + ly * VEC + (j % VEC);
+#pragma unroll
+      for (int i = 0; i < TM; ++i) {
+        const int64_t row = m0 + warp_m * WTM + (i / VEC) * 8 * VEC + lx * VEC + (i % VEC);
+        if (row < p.m && col < p.n && in_triangle(p.tri, row, col)) {
+          T* dst = C + col * p.ldc + row;
+          T v = p.alpha * get(acc, i, j);
+          if (use_beta) v += p.beta * *dst;
+          *dst = v;
         }
       }
     }
@@ -515,11 +565,12 @@ struct GemmKernel {
     int tm, tn;
     tile_coords(blockIdx.x, p.tiles_m, p.tiles_n, p.group_m, tm, tn);
     const int64_t m0 = (int64_t)tm * BM, n0 = (int64_t)tn * BN;
+    if (tile_outside_triangle(p.tri, m0, n0, BM, BN)) return;  // triangular update: nothing of this tile is stored
     const int m_valid = (int)min((int64_t)BM, p.m - m0), n_valid = (int)min((int64_t)BN, p.n - n0);
 
-    // element (m0, 0) of op(A) and (0, n0) of op(B)
-    const T* gA = TA ? p.A + m0 * p.lda : p.A + m0;
-    const T* gB = TB ? p.B + n0 : p.B + n0 * p.ldb;
+    // element (m0, 0) of op(A) and (0, n0) of op(B) of problem blockIdx.y of a strided batch
+    const T* gA = p.A + (int64_t)blockIdx.y * p.batch_a + (TA ? m0 * p.lda : m0);
+    const T* gB = p.B + (int64_t)blockIdx.y * p.batch_b + (TB ? n0 : n0 * p.ldb);
     const int64_t stepA = TA ? (int64_t)BK : (int64_t)BK * p.lda;  // advance by BK along k
     const int64_t stepB = TB ? (int64_t)BK * p.ldb : (int64_t)BK;
 
@@ -540,7 +591,7 @@ struct GemmKernel {
       for (int c = tid; c < BN * LPC; c += NT) {
         const int col = c / LPC, row = (c % LPC) * LINE;
         if (col < n_valid && row < m_valid) {
-          const T* ptr = p.C + (n0 + col) * p.ldc + m0 + row;
+          const T* ptr = p.C + (int64_t)blockIdx.y * p.batch_c + (n0 + col) * p.ldc + m0 + row;
           asm volatile("prefetch.global.L2 [%0];" ::"l"(ptr));
         }
       }
@@ -553,21 +604,21 @@ struct GemmKernel {
       T* dB = sB + slot * Micro::B_STAGE;
       if (k_valid == BK) {
         if (a_inside) {
-          stA.load_fast(dA);
+          stA.load_fast(dA, p.lda, tid);
         } else {
-          stA.load_edge(dA, m_valid, tid);
+          stA.load_edge(dA, p.lda, m_valid, tid);
         }
         if (b_inside) {
-          stB.load_fast(dB);
+          stB.load_fast(dB, p.ldb, tid);
         } else {
-          stB.load_edge(dB, n_valid, tid);
+          stB.load_edge(dB, p.ldb, n_valid, tid);
         }
       } else {
         StageA::load_general(dA, gA + kt * stepA, p.lda, m_valid, k_valid, tid);
         StageB::load_general(dB, gB + kt * stepB, p.ldb, n_valid, k_valid, tid);
       }
-      stA.advance();
-      stB.advance();
+      stA.advance(p.lda);
+      stB.advance(p.ldb);
     };
 
     // ramp-up: fill STAGES-1 slots (the first of the paper's three stages of the k-loop)
@@ -594,7 +645,12 @@ struct GemmKernel {
     cp_async_wait<0>();
 
     // drain: fused alpha/beta epilogue
-    Micro::epilogue(acc, p, m0, n0, warp_m, warp_n, lane);
+    T* Cb = p.C + (int64_t)blockIdx.y * p.batch_c;
+    if (tile_crosses_diagonal(p.tri, m0, n0, BM, BN)) {
+      Micro::epilogue_masked(acc, p, Cb, m0, n0, warp_m, warp_n, lane);
+    } else {
+      Micro::epilogue(acc, p, Cb, m0, n0, warp_m, warp_n, lane);
+    }
   }
 };
 

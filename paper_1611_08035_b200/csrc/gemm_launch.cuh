@@ -31,7 +31,8 @@ int launch_one(const GemmArgs<typename Kernel::T>& args, cudaStream_t stream) {
   }
   const long long tiles = (long long)args.tiles_m * args.tiles_n;
   if (tiles <= 0 || tiles > 0x7fffffffLL) return B2_ERR_LAUNCH;
-  kfn<<<(unsigned)tiles, Kernel::NT, Kernel::SMEM_BYTES, stream>>>(args);
+  const int batch = args.batch > 0 ? args.batch : 1;
+  kfn<<<dim3((unsigned)tiles, (unsigned)batch, 1), Kernel::NT, Kernel::SMEM_BYTES, stream>>>(args);
   return cudaGetLastError() == cudaSuccess ? B2_OK : B2_ERR_LAUNCH;
 }
 

@@ -91,6 +91,7 @@ struct GemmTmaKernel {
     int tm, tn;
     tile_coords(blockIdx.x, p.tiles_m, p.tiles_n, p.group_m, tm, tn);
     const int64_t m0 = (int64_t)tm * BM, n0 = (int64_t)tn * BN;
+    if (tile_outside_triangle(p.tri, m0, n0, BM, BN)) return;  // triangular update: nothing of this tile is stored
     const int KT = (int)((p.k + BK - 1) / BK);
 
     if (tid == 0) {
@@ -169,7 +170,11 @@ struct GemmTmaKernel {
       }
       return;
     }
-    Micro::epilogue(acc, p, m0, n0, warp_m, warp_n, lane);
+    if (tile_crosses_diagonal(p.tri, m0, n0, BM, BN)) {
+      Micro::epilogue_masked(acc, p, p.C, m0, n0, warp_m, warp_n, lane);
+    } else {
+      Micro::epilogue(acc, p, p.C, m0, n0, warp_m, warp_n, lane);
+    }
   }
 };
 
