@@ -41,7 +41,11 @@ def run_syrk(b2, oracle, kind, uplo, trans, n, k, alpha, beta, dist="uniform", s
     _, S = oracle.ref_gemm_hi(trans, "T" if trans == "N" else "N", n, n, k, alpha, A.numpy(), lda, A.numpy(), lda, beta,
                               C.numpy(), ldc)
     err = np.abs(g.astype(np.float64) - w.astype(np.float64))
-    assert np.all(err[tri] <= (2 * k * U[np.dtype(ndt)] * S.reshape(n, n))[tri])
+    bad = (err > 2 * k * U[np.dtype(ndt)] * S.reshape(n, n)) & tri
+    if bad.any():
+        where = np.argwhere(bad)
+        raise AssertionError(f"{int(bad.sum())} elements of the triangle exceed the bound; first (col, row): "
+                             f"{where[:8].tolist()}, got {g[bad][:4]}, want {w[bad][:4]}, old {C0[:, :n][bad][:4]}")
 
 
 @pytest.mark.parametrize("kind", ["d", "s"])
