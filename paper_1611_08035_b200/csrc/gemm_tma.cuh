@@ -156,6 +156,11 @@ struct GemmTmaKernel {
       }
       waited = kt + 1;
       Micro::compute(acc, sA + slot * Micro::A_STAGE, sB + slot * Micro::B_STAGE, warp_m, warp_n, lane);
+      // The fragment loads above went through the generic proxy; the refill of this slot is written by the
+      // async proxy.  Accesses to one location through two proxies are ordered only by a proxy fence, and the
+      // mbarrier hand-off alone does not supply it: without this fence the refill was observed (rarely, a
+      // few tiles in 65536) to land before a warp's last fragment loads of the slab it replaces.
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       __syncwarp();
       if (lane == 0) mbar_arrive(&empty[slot]);
     }

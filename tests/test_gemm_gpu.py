@@ -61,6 +61,35 @@ def test_config3_rank_k_update_sampled(b2, oracle, k):
     run_and_check(b2, oracle, "d", "N", "N", 16384, 16384, k, -1.0, 1.0, dist="normal", seed=3000 + k, cols=cols)
 
 
+@pytest.mark.parametrize("k", [64, 128])
+def test_rank_k_update_whole_matrix_every_staging(b2, oracle, k):
+    """The short-k shape launches 65536 short-lived CTAs, where a slot of the staging ring is recycled right
+    after the CTA starts: the place a producer/consumer hand-off error shows.  Integer data make the exact
+    result independent of the summation order, so every fp64 tensor-core variant must produce the same bits
+    over the WHOLE matrix, launch after launch; the oracle then checks a column sample of that result."""
+    m = n = 16384
+    A, lda, B, ldb, C, ldc = synth.gemm_inputs("N", "N", m, n, k, "int9", 3100 + k, torch.float64, device="cuda")
+    names = [b2.b2_variant_name(0, v) for v in range(nvariants(b2, "d"))]
+    first = None
+    for v, name in enumerate(names):
+        if "dmma" not in name:
+            continue
+        for rep in range(3 if "tma" in name else 1):
+            Cd = C.clone()
+            b2.b2_dgemm("N", "N", m, n, k, -1.0, A, lda, B, ldb, 1.0, Cd, ldc, variant=v)
+            assert b2.b2_device_status() == 0
+            if first is None:
+                first = Cd
+            else:
+                differing = int((Cd != first).sum())
+                assert differing == 0, f"{name}, launch {rep}: {differing} elements differ from {names[0]}"
+    cols = sample_columns(n, tile=64, extra=24, seed=k)
+    want = C.cpu().numpy()
+    oracle.ref_gemm("N", "N", m, n, k, -1.0, A.cpu().numpy(), lda, B.cpu().numpy(), ldb, 1.0, want, ldc, cols=cols)
+    got = first.cpu().numpy().reshape(n, ldc)[cols]
+    assert got.tobytes() == want.reshape(n, ldc)[cols].tobytes()
+
+
 @pytest.mark.parametrize("kind", ["d", "s"])
 @pytest.mark.parametrize("ta,tb", TRANS)
 def test_config4_fringe_and_transposes(b2, oracle, kind, ta, tb):
