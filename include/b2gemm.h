@@ -213,7 +213,10 @@ int b2_sgemm_tf32x3(char transa, char transb, int64_t m, int64_t n, int64_t k, f
  * dev_workspace is DEVICE memory of at least b2_gemm_host_workspace_bytes(...) bytes owned by
  * the caller.  The call copies the referenced parts of A and B (and C when beta != 0) to the
  * device, runs the same kernel as b2_dgemm / b2_sgemm, copies the m x n result back into C and
- * synchronises the stream before returning.  Argument numbering as b2_dgemm, workspace = 14.
+ * synchronises the stream before returning.  Copies and compute are pipelined over column panels of
+ * C on two helper streams that the library creates on its first such call on a device and keeps
+ * (no device memory is allocated); these calls are serialised among host threads.
+ * Argument numbering as b2_dgemm, workspace = 14.
  */
 size_t b2_gemm_host_workspace_bytes(int dtype, char transa, char transb, int64_t m, int64_t n, int64_t k);
 int b2_dgemm_host(char transa, char transb, int64_t m, int64_t n, int64_t k, double alpha, const double* A,

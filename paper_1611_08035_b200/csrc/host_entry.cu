@@ -1,5 +1,13 @@
 // Host-buffer forms of the real GEMM: copy the referenced parts of A, B (and C when beta != 0)
 // into the caller's device workspace, run the device entry point, copy the result back.
+//
+// The copies and the multiplication are pipelined over column panels of C: A goes up first, then the panels
+// of B (and of C when beta != 0) follow on a copy-in stream while the kernel works on the panels that have
+// arrived and a copy-out stream returns finished panels -- PCIe is full duplex, so the call takes about
+// max(copy time, compute time) instead of their sum.  The two helper streams and a few events are created on
+// the first call on a device and kept (no device memory is allocated); calls are serialised by a mutex.
+#include <mutex>
+
 #include "b2gemm.h"
 #include "entry.h"
 
@@ -27,6 +35,30 @@ HostPlan host_plan(int elem, char transa, char transb, int64_t m, int64_t n, int
   return p;
 }
 
+// Helper streams and events of the pipelined host-buffer calls, one set per device, created on first use.
+constexpr int kMaxPanels = 16;
+struct HostPipe {
+  cudaStream_t cin, cout;
+  cudaEvent_t start, a_ready, out_done, in[kMaxPanels], done[kMaxPanels];
+};
+HostPipe* host_pipe() {
+  static HostPipe pipes[64];
+  static bool ready[64] = {};
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  if (!ready[dev]) {
+    HostPipe& h = pipes[dev];
+    bool good = cudaStreamCreateWithFlags(&h.cin, cudaStreamNonBlocking) == cudaSuccess &&
+                cudaStreamCreateWithFlags(&h.cout, cudaStreamNonBlocking) == cudaSuccess;
+    auto ev = [&good](cudaEvent_t* e) { good = good && cudaEventCreateWithFlags(e, cudaEventDisableTiming) == cudaSuccess; };
+    ev(&h.start), ev(&h.a_ready), ev(&h.out_done);
+    for (int i = 0; i < kMaxPanels; ++i) ev(&h.in[i]), ev(&h.done[i]);
+    if (!good) return nullptr;
+    ready[dev] = true;
+  }
+  return &pipes[dev];
+}
+
 template <typename T>
 int gemm_host(char transa, char transb, int64_t m, int64_t n, int64_t k, T alpha, const T* A, int64_t lda, const T* B,
               int64_t ldb, T beta, T* C, int64_t ldc, void* ws, size_t ws_bytes, void* cuda_stream) {
@@ -43,21 +75,56 @@ int gemm_host(char transa, char transb, int64_t m, int64_t n, int64_t k, T alpha
   T* dB = reinterpret_cast<T*>(w + p.off_b);
   T* dC = reinterpret_cast<T*>(w + p.off_c);
   const size_t e = sizeof(T);
-  if (!scale_only) {
-    if (cudaMemcpy2DAsync(dA, p.lda_d * e, A, lda * e, p.ra * e, p.ca, cudaMemcpyHostToDevice, st) != cudaSuccess)
-      return B2_ERR_LAUNCH;
-    if (cudaMemcpy2DAsync(dB, p.ldb_d * e, B, ldb * e, p.rb * e, p.cb, cudaMemcpyHostToDevice, st) != cudaSuccess)
-      return B2_ERR_LAUNCH;
-  }
-  if (beta != T(0)) {
-    if (cudaMemcpy2DAsync(dC, p.ldc_d * e, C, ldc * e, m * e, n, cudaMemcpyHostToDevice, st) != cudaSuccess)
-      return B2_ERR_LAUNCH;
-  }
-  const int rc = gemm_entry<T>(B2_VARIANT_AUTO, transa, transb, m, n, k, alpha, dA, p.lda_d, dB, p.ldb_d, beta, dC,
-                               p.ldc_d, cuda_stream);
-  if (rc) return rc;
-  if (cudaMemcpy2DAsync(C, ldc * e, dC, p.ldc_d * e, m * e, n, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+
+  static std::mutex mu;
+  std::lock_guard<std::mutex> lock(mu);
+  HostPipe* hp = host_pipe();
+  if (!hp) return B2_ERR_LAUNCH;
+  auto ok = [](cudaError_t err) { return err == cudaSuccess; };
+
+  // column panels of C: at least 512 columns each, at most kMaxPanels, multiples of 64 columns
+  int64_t panels = n / 1024;
+  panels = panels < 1 ? 1 : (panels > kMaxPanels ? kMaxPanels : panels);
+  const int64_t width = ((n + panels - 1) / panels + 63) / 64 * 64;
+  const bool tb = !h_is_n(transb);
+
+  // both helper streams start after whatever the caller's stream has queued so far
+  if (!ok(cudaEventRecord(hp->start, st)) || !ok(cudaStreamWaitEvent(hp->cin, hp->start, 0)) ||
+      !ok(cudaStreamWaitEvent(hp->cout, hp->start, 0)))
     return B2_ERR_LAUNCH;
+  if (!scale_only) {
+    if (!ok(cudaMemcpy2DAsync(dA, p.lda_d * e, A, lda * e, p.ra * e, p.ca, cudaMemcpyHostToDevice, hp->cin)))
+      return B2_ERR_LAUNCH;
+  }
+  if (!ok(cudaEventRecord(hp->a_ready, hp->cin)) || !ok(cudaStreamWaitEvent(st, hp->a_ready, 0))) return B2_ERR_LAUNCH;
+  int np = 0;
+  for (int64_t j0 = 0; j0 < n; j0 += width, ++np) {
+    const int64_t nj = (n - j0) < width ? (n - j0) : width;
+    if (!scale_only) {
+      // panel of op(B): columns j0.. of a k x n matrix, or rows j0.. of an n x k matrix
+      const cudaError_t err =
+          tb ? cudaMemcpy2DAsync(dB + j0, p.ldb_d * e, B + j0, ldb * e, nj * e, p.cb, cudaMemcpyHostToDevice, hp->cin)
+             : cudaMemcpy2DAsync(dB + j0 * p.ldb_d, p.ldb_d * e, B + j0 * ldb, ldb * e, p.rb * e, nj,
+                                 cudaMemcpyHostToDevice, hp->cin);
+      if (!ok(err)) return B2_ERR_LAUNCH;
+    }
+    if (beta != T(0)) {
+      if (!ok(cudaMemcpy2DAsync(dC + j0 * p.ldc_d, p.ldc_d * e, C + j0 * ldc, ldc * e, m * e, nj, cudaMemcpyHostToDevice,
+                                hp->cin)))
+        return B2_ERR_LAUNCH;
+    }
+    if (!ok(cudaEventRecord(hp->in[np], hp->cin)) || !ok(cudaStreamWaitEvent(st, hp->in[np], 0))) return B2_ERR_LAUNCH;
+    const T* dBj = tb ? dB + j0 : dB + j0 * p.ldb_d;
+    const int rc = gemm_entry<T>(B2_VARIANT_AUTO, transa, transb, m, nj, k, alpha, dA, p.lda_d, dBj, p.ldb_d, beta,
+                                 dC + j0 * p.ldc_d, p.ldc_d, cuda_stream);
+    if (rc) return rc;
+    if (!ok(cudaEventRecord(hp->done[np], st)) || !ok(cudaStreamWaitEvent(hp->cout, hp->done[np], 0)))
+      return B2_ERR_LAUNCH;
+    if (!ok(cudaMemcpy2DAsync(C + j0 * ldc, ldc * e, dC + j0 * p.ldc_d, p.ldc_d * e, m * e, nj, cudaMemcpyDeviceToHost,
+                              hp->cout)))
+      return B2_ERR_LAUNCH;
+  }
+  if (!ok(cudaEventRecord(hp->out_done, hp->cout)) || !ok(cudaStreamWaitEvent(st, hp->out_done, 0))) return B2_ERR_LAUNCH;
   return cudaStreamSynchronize(st) == cudaSuccess ? B2_OK : B2_ERR_LAUNCH;
 }
 
