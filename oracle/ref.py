@@ -152,22 +152,23 @@ def ref_gemm_hi(transa, transb, m, n, k, alpha, A, lda, B, ldb, beta, C, ldc, co
     return Chi, S
 
 
-def ref_zgemm_4m(transa, transb, m, n, k, alpha, A, lda, B, ldb, beta, C, ldc) -> None:
-    """Complex GEMM from four real-oracle calls on split planes (4M); C complex128 flat, updated in place.
+def _split_planes(transa, transb, alpha, beta, A, B, C):
+    """Real and imaginary planes for the 4M / 3M step oracles: A' = alpha*op-conjugated A, B, beta*C.
 
-    A' = alpha*A is formed elementwise in complex arithmetic (each component rounded once), then
-        Cr = A'r*Br - A'i*Bi + (beta*C)r,     Ci = A'r*Bi + A'i*Br + (beta*C)i,
-    each right-hand side evaluated as two real GEMM calls: (alpha=1, beta=0 or 1) followed by
-    (alpha=-1 or +1, beta=1).  With beta == 0 the old C is not read.
-    """
+    A conjugate transpose becomes a plain transpose of the conjugated matrix (negating the imaginary plane is
+    exact); returns (apr, api, br, bi, cr, ci, first_beta, ta, tb) with ta/tb the real transposes to use."""
     alpha, beta = complex(alpha), complex(beta)
     _flat(A, np.complex128), _flat(B, np.complex128), _flat(C, np.complex128)
     Av = A.view(np.float64)
     ar, ai = Av[0::2], Av[1::2]
+    if transa in "Cc":
+        ai = -ai
     apr = np.ascontiguousarray(alpha.real * ar - alpha.imag * ai)
     api = np.ascontiguousarray(alpha.real * ai + alpha.imag * ar)
     Bv = B.view(np.float64)
     br, bi = np.ascontiguousarray(Bv[0::2]), np.ascontiguousarray(Bv[1::2])
+    if transb in "Cc":
+        bi = -bi
     Cv = C.view(np.float64)
     cr0, ci0 = Cv[0::2].copy(), Cv[1::2].copy()
     if beta == 0:
@@ -176,15 +177,58 @@ def ref_zgemm_4m(transa, transb, m, n, k, alpha, A, lda, B, ldb, beta, C, ldc) -
         cr = np.ascontiguousarray(beta.real * cr0 - beta.imag * ci0)
         ci = np.ascontiguousarray(beta.real * ci0 + beta.imag * cr0)
         first_beta = 1.0
-    ref_gemm(transa, transb, m, n, k, 1.0, apr, lda, br, ldb, first_beta, cr, ldc)
-    ref_gemm(transa, transb, m, n, k, -1.0, api, lda, bi, ldb, 1.0, cr, ldc)
-    ref_gemm(transa, transb, m, n, k, 1.0, apr, lda, bi, ldb, first_beta, ci, ldc)
-    ref_gemm(transa, transb, m, n, k, 1.0, api, lda, br, ldb, 1.0, ci, ldc)
-    # write back only the m x n entries the operation owns
-    for j in range(n):
+    ta = "N" if transa in "Nn" else "T"
+    tb = "N" if transb in "Nn" else "T"
+    return apr, api, br, bi, cr, ci, first_beta, ta, tb
+
+
+def _store_planes(C, cr, ci, m, n, ldc):
+    Cv = C.view(np.float64)
+    for j in range(n):  # write back only the m x n entries the operation owns
         s = slice(j * ldc, j * ldc + m)
         Cv[0::2][s] = cr[s]
         Cv[1::2][s] = ci[s]
+
+
+def ref_zgemm_4m(transa, transb, m, n, k, alpha, A, lda, B, ldb, beta, C, ldc) -> None:
+    """Complex GEMM from four real-oracle calls on split planes (4M); C complex128 flat, updated in place.
+
+    A' = alpha*A is formed elementwise in complex arithmetic (each component rounded once), then
+        Cr = A'r*Br - A'i*Bi + (beta*C)r,     Ci = A'r*Bi + A'i*Br + (beta*C)i,
+    each right-hand side evaluated as two real GEMM calls: (alpha=1, beta=0 or 1) followed by
+    (alpha=-1 or +1, beta=1).  With beta == 0 the old C is not read.  Conjugate transposes negate the
+    imaginary plane of that operand first.
+    """
+    apr, api, br, bi, cr, ci, first_beta, ta, tb = _split_planes(transa, transb, alpha, beta, A, B, C)
+    ref_gemm(ta, tb, m, n, k, 1.0, apr, lda, br, ldb, first_beta, cr, ldc)
+    ref_gemm(ta, tb, m, n, k, -1.0, api, lda, bi, ldb, 1.0, cr, ldc)
+    ref_gemm(ta, tb, m, n, k, 1.0, apr, lda, bi, ldb, first_beta, ci, ldc)
+    ref_gemm(ta, tb, m, n, k, 1.0, api, lda, br, ldb, 1.0, ci, ldc)
+    _store_planes(C, cr, ci, m, n, ldc)
+
+
+def ref_zgemm_3m(transa, transb, m, n, k, alpha, A, lda, B, ldb, beta, C, ldc) -> None:
+    """Complex GEMM from three real products (3M), the steps in this order; C complex128 flat, updated in place.
+
+        A' = alpha*A (as in 4M);  As = A'r + A'i,  Bs = Br + Bi     (one rounding per element)
+        T1 = A'r*Br,  T2 = A'i*Bi                                    (real GEMMs, beta = 0)
+        Cr = ((beta*C)r + T1) - T2
+        Ci = (((beta*C)i - T1) - T2) + As*Bs                         (last step: real GEMM with beta = 1)
+
+    The imaginary part is the difference of larger numbers, so its error is bounded relative to
+    sum (|Ar|+|Ai|)(|Br|+|Bi|), not to the magnitude of the imaginary products alone.
+    """
+    apr, api, br, bi, cr, ci, first_beta, ta, tb = _split_planes(transa, transb, alpha, beta, A, B, C)
+    a_sum = np.ascontiguousarray(apr + api)
+    b_sum = np.ascontiguousarray(br + bi)
+    t1 = np.zeros_like(cr)
+    t2 = np.zeros_like(cr)
+    ref_gemm(ta, tb, m, n, k, 1.0, apr, lda, br, ldb, 0.0, t1, ldc)
+    ref_gemm(ta, tb, m, n, k, 1.0, api, lda, bi, ldb, 0.0, t2, ldc)
+    cr = (cr + t1) - t2
+    ci = np.ascontiguousarray((ci - t1) - t2)
+    ref_gemm(ta, tb, m, n, k, 1.0, a_sum, lda, b_sum, ldb, 1.0, ci, ldc)
+    _store_planes(C, cr, ci, m, n, ldc)
 
 
 def tf32_round(x: float) -> float:

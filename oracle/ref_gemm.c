@@ -35,6 +35,7 @@
 
 static int is_trans(char t) { return t == 'T' || t == 't' || t == 'C' || t == 'c'; }
 static int is_notrans(char t) { return t == 'N' || t == 'n'; }
+static int is_conj(char t) { return t == 'C' || t == 'c'; } /* complex data only; for real data 'C' is 'T' */
 
 /* BLAS argument check; returns 0 or the 1-based index of the first illegal argument. */
 static int check_args(char ta, char tb, int64_t m, int64_t n, int64_t k, int64_t lda, int64_t ldb, int64_t ldc) {
@@ -131,18 +132,19 @@ DEFINE_REF_GEMM_HI(ref_sgemm_hi, float, double, fabs)
 /*
  * Complex double GEMM by direct complex arithmetic (interleaved re,im; ld in complex
  * elements).  Each term is the textbook product (ar*br - ai*bi, ar*bi + ai*br) added to the
- * running sum; the epilogue is the complex alpha*acc + beta*C.  transa/transb: N or T
- * (plain transpose; the conjugate transpose 'C' is rejected here).
+ * running sum; the epilogue is the complex alpha*acc + beta*C.  transa/transb: N, T (plain
+ * transpose) or C (conjugate transpose: the transposed element with its imaginary part
+ * negated).
  * The paper names complex GEMM only as a consumer of the real kernel (Abstract).
  */
 int ref_zgemm(char transa, char transb, int64_t m, int64_t n, int64_t k, const double* alpha, const double* A,
               int64_t lda, const double* B, int64_t ldb, const double* beta, double* C, int64_t ldc,
               const int64_t* cols, int64_t ncols) {
-  if (transa == 'C' || transa == 'c') return -1;
-  if (transb == 'C' || transb == 'c') return -2;
   int bad = check_args(transa, transb, m, n, k, lda, ldb, ldc);
   if (bad) return -bad;
   if (m == 0 || n == 0) return 0;
+  /* op(X) = X^H for 'C': the element is read transposed and its imaginary part negated (exact) */
+  const double ca = is_conj(transa) ? -1.0 : 1.0, cb = is_conj(transb) ? -1.0 : 1.0;
   const double alr = alpha[0], ali = alpha[1], ber = beta[0], bei = beta[1];
   const int alpha0 = (alr == 0.0 && ali == 0.0), beta0 = (ber == 0.0 && bei == 0.0);
   if ((alpha0 || k == 0) && ber == 1.0 && bei == 0.0) return 0;
@@ -157,8 +159,9 @@ int ref_zgemm(char transa, char transb, int64_t m, int64_t n, int64_t k, const d
         for (int64_t p = 0; p < k; ++p) {
           const double* a = ta ? &A[2 * (p + i * lda)] : &A[2 * (i + p * lda)];
           const double* b = tb ? &B[2 * (j + p * ldb)] : &B[2 * (p + j * ldb)];
-          const double pr = a[0] * b[0] - a[1] * b[1];
-          const double pi = a[0] * b[1] + a[1] * b[0];
+          const double are = a[0], aim = ca * a[1], bre = b[0], bim = cb * b[1];
+          const double pr = are * bre - aim * bim;
+          const double pi = are * bim + aim * bre;
           sr = sr + pr;
           si = si + pi;
         }
@@ -187,11 +190,10 @@ int ref_zgemm(char transa, char transb, int64_t m, int64_t n, int64_t k, const d
 int ref_zgemm_hi(char transa, char transb, int64_t m, int64_t n, int64_t k, const double* alpha, const double* A,
                  int64_t lda, const double* B, int64_t ldb, const double* beta, const double* C, int64_t ldc,
                  double* Chi, double* S, int64_t ldo, const int64_t* cols, int64_t ncols) {
-  if (transa == 'C' || transa == 'c') return -1;
-  if (transb == 'C' || transb == 'c') return -2;
   int bad = check_args(transa, transb, m, n, k, lda, ldb, ldc);
   if (bad) return -bad;
   if (ldo < (m > 1 ? m : 1)) return -16;
+  const double ca = is_conj(transa) ? -1.0 : 1.0, cb = is_conj(transb) ? -1.0 : 1.0;
   if (m == 0 || n == 0) return 0;
   const long double alr = alpha[0], ali = alpha[1], ber = beta[0], bei = beta[1];
   const int alpha0 = (alr == 0 && ali == 0), beta0 = (ber == 0 && bei == 0);
@@ -206,7 +208,7 @@ int ref_zgemm_hi(char transa, char transb, int64_t m, int64_t n, int64_t k, cons
         for (int64_t p = 0; p < k; ++p) {
           const double* a = ta ? &A[2 * (p + i * lda)] : &A[2 * (i + p * lda)];
           const double* b = tb ? &B[2 * (j + p * ldb)] : &B[2 * (p + j * ldb)];
-          const long double ar = a[0], ai = a[1], br = b[0], bi = b[1];
+          const long double ar = a[0], ai = ca * a[1], br = b[0], bi = cb * b[1];
           sr += ar * br - ai * bi;
           si += ar * bi + ai * br;
           mag += (fabsl(ar) + fabsl(ai)) * (fabsl(br) + fabsl(bi));

@@ -339,7 +339,82 @@ def test_complex_quick_returns(oracle):
     oracle.ref_gemm("N", "N", m, n, k, 1 + 0j, store(A2, m, np.nan), m, store(B2, k, np.nan), k, 0j, C, m)
     assert np.all(np.isfinite(unstore(C, m, n, m)))
     with pytest.raises(ValueError):
-        oracle.ref_gemm("C", "N", m, n, k, 1 + 0j, store(A2, m, np.nan), m, store(B2, k, np.nan), k, 0j, C, m)
+        oracle.ref_gemm("X", "N", m, n, k, 1 + 0j, store(A2, m, np.nan), m, store(B2, k, np.nan), k, 0j, C, m)
+
+
+def _zint(rng, shape):
+    return (rng.integers(-4, 5, shape) + 1j * rng.integers(-4, 5, shape)).astype(np.complex128)
+
+
+def _zop(X, t):
+    return X if t == "N" else (X.T if t == "T" else X.conj().T)
+
+
+def test_conjugate_transposes_of_the_complex_oracle(oracle):
+    """'C' pinned four ways: numpy's X.conj().T on exact integer data (all nine op pairs, direct, 4M and 3M);
+    'C' on X equals 'T' on conj(X) bit for bit (negation is exact); the Hermitian identity
+    (A^H B)^H = B^H A bit for bit (same products, multiplication commutes, the imaginary parts are exact
+    negatives); and the diagonal of A^H A has imaginary part exactly zero and a non-negative real part."""
+    rng = np.random.default_rng(21)
+    m, n, k = 6, 5, 7
+    for ta in "NTC":
+        for tb in "NTC":
+            ra, ca = (m, k) if ta == "N" else (k, m)
+            rb, cb = (k, n) if tb == "N" else (n, k)
+            A2, B2, C2 = _zint(rng, (ra, ca)), _zint(rng, (rb, cb)), _zint(rng, (m, n))
+            alpha, beta = 2 - 1j, 0.5 + 0.5j
+            want = alpha * (_zop(A2, ta) @ _zop(B2, tb)) + beta * C2
+            A, B = store(A2, ra + 1, np.nan), store(B2, rb + 3, np.nan)
+            for fn in (oracle.ref_gemm, oracle.ref_zgemm_4m, oracle.ref_zgemm_3m):
+                C = store(C2, m + 2, SENTINEL)
+                fn(ta, tb, m, n, k, alpha, A, ra + 1, B, rb + 3, beta, C, m + 2)
+                assert np.array_equal(unstore(C, m, n, m + 2), want), (ta, tb, fn.__name__)
+                assert np.all(padding(C, m, n, m + 2).real == SENTINEL)
+    # general data: C on X == T on conj(X), bitwise
+    A2 = rng.uniform(-1, 1, (k, m)) + 1j * rng.uniform(-1, 1, (k, m))
+    B2 = rng.uniform(-1, 1, (k, n)) + 1j * rng.uniform(-1, 1, (k, n))
+    C2 = rng.uniform(-1, 1, (m, n)) + 1j * rng.uniform(-1, 1, (m, n))
+    X, Y = store(C2, m, SENTINEL), store(C2, m, SENTINEL)
+    oracle.ref_gemm("C", "N", m, n, k, 0.7 - 0.2j, store(A2, k, np.nan), k, store(B2, k, np.nan), k, 0.3j, X, m)
+    oracle.ref_gemm("T", "N", m, n, k, 0.7 - 0.2j, store(A2.conj(), k, np.nan), k, store(B2, k, np.nan), k, 0.3j, Y, m)
+    assert bits_equal(X, Y)
+    # Hermitian identity, bitwise
+    X, Y = store(np.zeros((m, n), complex), m, SENTINEL), store(np.zeros((n, m), complex), n, SENTINEL)
+    oracle.ref_gemm("C", "N", m, n, k, 1 + 0j, store(A2, k, np.nan), k, store(B2, k, np.nan), k, 0j, X, m)
+    oracle.ref_gemm("C", "N", n, m, k, 1 + 0j, store(B2, k, np.nan), k, store(A2, k, np.nan), k, 0j, Y, n)
+    assert bits_equal(unstore(X, m, n, m), unstore(Y, n, m, n).conj().T)
+    # Gram matrix
+    G = store(np.zeros((m, m), complex), m, SENTINEL)
+    oracle.ref_gemm("C", "N", m, m, k, 1 + 0j, store(A2, k, np.nan), k, store(A2, k, np.nan), k, 0j, G, m)
+    d = np.diag(unstore(G, m, m, m))
+    assert np.all(d.imag == 0.0) and np.all(d.real > 0.0)
+    assert np.allclose(d.real, np.sum(np.abs(A2) ** 2, axis=0), rtol=1e-14)
+
+
+def test_3m_steps_against_the_definition(oracle):
+    """3M against direct complex arithmetic on general data: both components within 2*(3k+6)*u*S of the wide
+    result (S = sum (|Ar|+|Ai|)(|Br|+|Bi|) scaled by |alpha| plus the beta term), and the real component, which
+    3M computes exactly as 4M does, bitwise equal to 4M's."""
+    rng = np.random.default_rng(22)
+    m, n, k = 24, 20, 65
+    for ta in "NC":
+        for tb in "NT":
+            ra, ca = (m, k) if ta == "N" else (k, m)
+            rb, cb = (k, n) if tb == "N" else (n, k)
+            A2 = rng.uniform(-1, 1, (ra, ca)) + 1j * rng.uniform(-1, 1, (ra, ca))
+            B2 = rng.uniform(-1, 1, (rb, cb)) + 1j * rng.uniform(-1, 1, (rb, cb))
+            C2 = rng.uniform(-1, 1, (m, n)) + 1j * rng.uniform(-1, 1, (m, n))
+            alpha, beta = (1 + 0.5j), (0.25 - 0.75j)
+            A, B = store(A2, ra, np.nan), store(B2, rb, np.nan)
+            C3, C4, C0 = store(C2, m, SENTINEL), store(C2, m, SENTINEL), store(C2, m, SENTINEL)
+            hi, S = oracle.ref_gemm_hi(ta, tb, m, n, k, alpha, A, ra, B, rb, beta, C0, m)
+            oracle.ref_zgemm_3m(ta, tb, m, n, k, alpha, A, ra, B, rb, beta, C3, m)
+            oracle.ref_zgemm_4m(ta, tb, m, n, k, alpha, A, ra, B, rb, beta, C4, m)
+            bound = 2 * (3 * k + 6) * 2.0 ** -53 * unstore(S, m, n, m)
+            d = unstore(C3, m, n, m) - unstore(hi, m, n, m)
+            assert np.all(np.abs(d.real) <= bound) and np.all(np.abs(d.imag) <= bound)
+            assert bits_equal(unstore(C3, m, n, m).real.copy(), unstore(C4, m, n, m).real.copy())
+            assert not bits_equal(unstore(C3, m, n, m).imag.copy(), unstore(C4, m, n, m).imag.copy())
 
 
 def test_padding_of_operands_is_never_used(oracle):
