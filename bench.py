@@ -215,6 +215,13 @@ def other_configs(b2, device):
     g = quick_gflops(lambda: b2.b2_zgemm4m("N", "N", m, n, k, 1 + 0.5j, A, m, B, k, 0j, C, m, ws), 8.0 * m * n * k,
                      iters=2, warm=2)
     out.append({"workload": "zgemm4m_nn_4096", "gflops": round(g, 1), "frac_of_peak": round(g / 1e3 / FP64_PEAK_TFLOPS, 4)})
+    del ws
+    ws = torch.empty(b2.b2_zgemm3m_workspace_bytes("N", "N", m, n, k), dtype=torch.uint8, device=device)
+    g = quick_gflops(lambda: b2.b2_zgemm3m("N", "N", m, n, k, 1 + 0.5j, A, m, B, k, 0j, C, m, ws), 8.0 * m * n * k,
+                     iters=2, warm=2)
+    out.append({"workload": "zgemm3m_nn_4096", "gflops": round(g, 1),
+                "note": "8*m*n*k flops counted although 3M executes 6*m*n*k: the figure may exceed the FP64 peak",
+                "frac_of_peak_executed": round(0.75 * g / 1e3 / FP64_PEAK_TFLOPS, 4)})
     return out
 
 

@@ -120,13 +120,29 @@ int b2_gemm_query_config(int dtype, char transa, char transb, int64_t m, int64_t
  * elements) built from four real-kernel launches ("4M"): the paper names complex GEMM only
  * as a consumer of the real kernel (Abstract).  With A' = alpha*A rounded once per component,
  *     Cr = A'r*Br - A'i*Bi + (beta*C)r,   Ci = A'r*Bi + A'i*Br + (beta*C)i.
- * alpha and beta point to HOST {re, im} pairs.  transa/transb accept N and T (C, the
- * conjugate transpose, is rejected with -1/-2).  workspace is DEVICE memory of at least
+ * alpha and beta point to HOST {re, im} pairs.  transa/transb accept N, T and C (conjugate
+ * transpose: the operand's imaginary plane is negated while it is split, then the real
+ * kernels see a plain transpose).  workspace is DEVICE memory of at least
  * b2_zgemm4m_workspace_bytes(...) bytes, 256-byte aligned, owned by the caller; its contents
  * are overwritten.  Argument numbering as above with workspace = 14.
  */
 size_t b2_zgemm4m_workspace_bytes(char transa, char transb, int64_t m, int64_t n, int64_t k);
 int b2_zgemm4m(char transa, char transb, int64_t m, int64_t n, int64_t k, const double alpha[2], const void* A,
+               int64_t lda, const void* B, int64_t ldb, const double beta[2], void* C, int64_t ldc,
+               void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * The same operation from THREE real products ("3M") instead of four:
+ *     T1 = A'r*Br,  T2 = A'i*Bi,  T3 = (A'r + A'i)*(Br + Bi),
+ *     Cr = ((beta*C)r + T1) - T2,   Ci = (((beta*C)i - T1) - T2) + T3.
+ * A quarter less arithmetic; the imaginary part is a difference of larger numbers, so each
+ * component's error is bounded relative to sum_p (|Ar|+|Ai|)_ip (|Br|+|Bi|)_pj rather than to
+ * the component's own products (not in the paper, which names complex GEMM only as a
+ * consumer of the real kernel).  Arguments, transposes, quick returns, error returns and
+ * workspace rules as for b2_zgemm4m, with b2_zgemm3m_workspace_bytes(...) bytes (nine planes).
+ */
+size_t b2_zgemm3m_workspace_bytes(char transa, char transb, int64_t m, int64_t n, int64_t k);
+int b2_zgemm3m(char transa, char transb, int64_t m, int64_t n, int64_t k, const double alpha[2], const void* A,
                int64_t lda, const void* B, int64_t ldb, const double beta[2], void* C, int64_t ldc,
                void* workspace, size_t workspace_bytes, void* cuda_stream);
 

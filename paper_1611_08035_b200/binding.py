@@ -36,6 +36,10 @@ _SIGNATURES = {
     "b2_zgemm4m": (c_int, [c_char, c_char, c_int64, c_int64, c_int64, ctypes.POINTER(c_double), c_void_p, c_int64,
                            c_void_p, c_int64, ctypes.POINTER(c_double), c_void_p, c_int64, c_void_p, c_size_t,
                            c_void_p]),
+    "b2_zgemm3m_workspace_bytes": (c_size_t, [c_char, c_char, c_int64, c_int64, c_int64]),
+    "b2_zgemm3m": (c_int, [c_char, c_char, c_int64, c_int64, c_int64, ctypes.POINTER(c_double), c_void_p, c_int64,
+                           c_void_p, c_int64, ctypes.POINTER(c_double), c_void_p, c_int64, c_void_p, c_size_t,
+                           c_void_p]),
     "b2_zgemm4m_static": (c_int, [c_char, c_char, c_int64, c_int64, c_int64, ctypes.POINTER(c_double), c_void_p, c_int64,
                                   c_void_p, c_int64, ctypes.POINTER(c_double), c_void_p, c_int64, c_void_p]),
     "b2_dsyrk": (c_int, [c_char, c_char, c_int64, c_int64, c_double, c_void_p, c_int64, c_double, c_void_p, c_int64,
@@ -178,6 +182,25 @@ def b2_zgemm4m(transa, transb, m, n, k, alpha, A, lda, B, ldb, beta, C, ldc, wor
                           _ptr(workspace), wbytes, _stream())
     if check:
         _check("b2_zgemm4m", rc)
+    return rc
+
+
+def b2_zgemm3m_workspace_bytes(transa, transb, m, n, k) -> int:
+    return lib().b2_zgemm3m_workspace_bytes(_tr(transa), _tr(transb), m, n, k)
+
+
+def b2_zgemm3m(transa, transb, m, n, k, alpha, A, lda, B, ldb, beta, C, ldc, workspace, check=True) -> int:
+    """Complex128 GEMM from three real-kernel launches (3M); same arguments as b2_zgemm4m."""
+    for t in (A, B, C):
+        if t is not None and (t.dtype != torch.complex128 or not t.is_cuda):
+            raise TypeError("b2_zgemm3m takes complex128 CUDA tensors")
+    al = (c_double * 2)(complex(alpha).real, complex(alpha).imag)
+    be = (c_double * 2)(complex(beta).real, complex(beta).imag)
+    wbytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    rc = lib().b2_zgemm3m(_tr(transa), _tr(transb), m, n, k, al, _ptr(A), lda, _ptr(B), ldb, be, _ptr(C), ldc,
+                          _ptr(workspace), wbytes, _stream())
+    if check:
+        _check("b2_zgemm3m", rc)
     return rc
 
 

@@ -1,4 +1,4 @@
-// Complex double GEMM assembled from four launches of the real kernel (4M).
+// Complex double GEMM assembled from four launches of the real kernel (4M), or three (3M).
 //
 // The paper treats complex GEMM only as a consumer of the real kernel (Abstract); the
 // decomposition used here is the textbook one on split real/imaginary planes:
@@ -14,13 +14,17 @@ namespace {
 
 // planes[0] = alpha_r*re - alpha_i*im, planes[1] = alpha_r*im + alpha_i*re of a rows x cols
 // interleaved complex matrix with leading dimension ld (complex elements); plane pitch ldp.
+// conj: the element is conjugated first (a conjugate transpose = plain transpose of these planes).
+// Ps != nullptr: also the plane of sums planes[0] + planes[1] (the third operand of 3M).
 __global__ void zsplit_scale_kernel(int64_t rows, int64_t cols, const double2* __restrict__ X, int64_t ld, double sr,
-                                    double si, double* __restrict__ Pr, double* __restrict__ Pi, int64_t ldp) {
+                                    double si, bool conj, double* __restrict__ Pr, double* __restrict__ Pi,
+                                    double* __restrict__ Ps, int64_t ldp) {
   const int64_t total = rows * cols;
   for (int64_t idx = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; idx < total;
        idx += (int64_t)gridDim.x * blockDim.x) {
     const int64_t r = idx % rows, c = idx / rows;
-    const double2 v = X[r + c * ld];
+    double2 v = X[r + c * ld];
+    if (conj) v.y = -v.y;
     double pr = v.x, pi = v.y;
     if (!(sr == 1.0 && si == 0.0)) {
       pr = sr * v.x - si * v.y;
@@ -28,6 +32,28 @@ __global__ void zsplit_scale_kernel(int64_t rows, int64_t cols, const double2* _
     }
     Pr[r + c * ldp] = pr;
     Pi[r + c * ldp] = pi;
+    if (Ps) Ps[r + c * ldp] = pr + pi;
+  }
+}
+
+// 3M: C := ((beta*C)r + T1 - T2,  ((beta*C)i - T1 - T2) + T3), the additions in exactly this order;
+// beta == 0: C is not read.
+__global__ void zmerge3m_kernel(int64_t rows, int64_t cols, const double* __restrict__ T1,
+                                const double* __restrict__ T2, const double* __restrict__ T3, int64_t ldp, double br,
+                                double bi, double2* __restrict__ X, int64_t ld) {
+  const int64_t total = rows * cols;
+  const bool zero = (br == 0.0 && bi == 0.0);
+  for (int64_t idx = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; idx < total;
+       idx += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t r = idx % rows, c = idx / rows;
+    double cr = 0.0, ci = 0.0;
+    if (!zero) {
+      const double2 v = X[r + c * ld];
+      cr = br * v.x - bi * v.y;
+      ci = br * v.y + bi * v.x;
+    }
+    const double t1 = T1[r + c * ldp], t2 = T2[r + c * ldp], t3 = T3[r + c * ldp];
+    X[r + c * ld] = make_double2((cr + t1) - t2, ((ci - t1) - t2) + t3);
   }
 }
 
@@ -69,10 +95,14 @@ struct Plan {
   int64_t ra, ca, rb, cb;     // stored rows/cols of A and B
   int64_t lpa, lpb, lpc;      // plane pitches (even, so plane columns are 16-byte aligned)
   size_t off[6], total;       // byte offsets of A'r, A'i, Br, Bi, Cr, Ci
+  size_t sa, sb, sc;          // bytes of one plane of A, B, C
 };
 
 bool is_n(char c) { return c == 'N' || c == 'n'; }
 bool is_t(char c) { return c == 'T' || c == 't'; }
+bool is_c(char c) { return c == 'C' || c == 'c'; }
+bool is_op(char c) { return is_n(c) || is_t(c) || is_c(c); }
+char real_op(char c) { return is_n(c) ? 'N' : 'T'; }  // the transpose the real kernels see
 
 Plan make_plan(char transa, char transb, int64_t m, int64_t n, int64_t k) {
   Plan p;
@@ -86,6 +116,7 @@ Plan make_plan(char transa, char transb, int64_t m, int64_t n, int64_t k) {
   p.off[0] = 0, p.off[1] = sa, p.off[2] = 2 * sa, p.off[3] = 2 * sa + sb, p.off[4] = 2 * sa + 2 * sb;
   p.off[5] = p.off[4] + sc;
   p.total = p.off[5] + sc;
+  p.sa = sa, p.sb = sb, p.sc = sc;
   return p;
 }
 
@@ -94,7 +125,7 @@ Plan make_plan(char transa, char transb, int64_t m, int64_t n, int64_t k) {
 
 extern "C" size_t b2_zgemm4m_workspace_bytes(char transa, char transb, int64_t m, int64_t n, int64_t k) {
   using namespace b2;
-  if ((!is_n(transa) && !is_t(transa)) || (!is_n(transb) && !is_t(transb)) || m < 0 || n < 0 || k < 0) return 0;
+  if (!is_op(transa) || !is_op(transb) || m < 0 || n < 0 || k < 0) return 0;
   return make_plan(transa, transb, m, n, k).total;
 }
 
@@ -102,8 +133,8 @@ extern "C" int b2_zgemm4m(char transa, char transb, int64_t m, int64_t n, int64_
                           const void* A, int64_t lda, const void* B, int64_t ldb, const double beta[2], void* C,
                           int64_t ldc, void* workspace, size_t workspace_bytes, void* cuda_stream) {
   using namespace b2;
-  if (!is_n(transa) && !is_t(transa)) return -1;  // conjugate transpose is not offered
-  if (!is_n(transb) && !is_t(transb)) return -2;
+  if (!is_op(transa)) return -1;
+  if (!is_op(transb)) return -2;
   if (!alpha) return -6;
   if (!beta) return -11;
   const double ar = alpha[0], ai = alpha[1], br = beta[0], bi = beta[1];
@@ -131,14 +162,15 @@ extern "C" int b2_zgemm4m(char transa, char transb, int64_t m, int64_t n, int64_
   double* Ci = reinterpret_cast<double*>(w + p.off[5]);
 
   zsplit_scale_kernel<<<grid_for(p.ra * p.ca), 256, 0, st>>>(p.ra, p.ca, static_cast<const double2*>(A), lda, ar, ai,
-                                                           Apr, Api, p.lpa);
+                                                           is_c(transa), Apr, Api, nullptr, p.lpa);
   zsplit_scale_kernel<<<grid_for(p.rb * p.cb), 256, 0, st>>>(p.rb, p.cb, static_cast<const double2*>(B), ldb, 1.0,
-                                                           0.0, Br, Bi, p.lpb);
+                                                           0.0, is_c(transb), Br, Bi, nullptr, p.lpb);
   double first_beta = 0.0;
   if (!beta0) {
-    zsplit_scale_kernel<<<grid_for(m * n), 256, 0, st>>>(m, n, Cz, ldc, br, bi, Cr, Ci, p.lpc);
+    zsplit_scale_kernel<<<grid_for(m * n), 256, 0, st>>>(m, n, Cz, ldc, br, bi, false, Cr, Ci, nullptr, p.lpc);
     first_beta = 1.0;
   }
+  transa = real_op(transa), transb = real_op(transb);
   if (cudaGetLastError() != cudaSuccess) return B2_ERR_LAUNCH;
   int rc;
   // Cr = A'r*Br + (beta*C)r ; Cr -= A'i*Bi
@@ -155,6 +187,64 @@ extern "C" int b2_zgemm4m(char transa, char transb, int64_t m, int64_t n, int64_
   return cudaGetLastError() == cudaSuccess ? B2_OK : B2_ERR_LAUNCH;
 }
 
+// ---- 3M: three real products instead of four ----------------------------------------------------
+// Planes in the workspace: A'r, A'i, A'r+A'i | Br, Bi, Br+Bi | T1, T2, T3 (m x n each).
+extern "C" size_t b2_zgemm3m_workspace_bytes(char transa, char transb, int64_t m, int64_t n, int64_t k) {
+  using namespace b2;
+  if (!is_op(transa) || !is_op(transb) || m < 0 || n < 0 || k < 0) return 0;
+  const Plan p = make_plan(transa, transb, m, n, k);
+  return 3 * (p.sa + p.sb + p.sc);
+}
+
+extern "C" int b2_zgemm3m(char transa, char transb, int64_t m, int64_t n, int64_t k, const double alpha[2],
+                          const void* A, int64_t lda, const void* B, int64_t ldb, const double beta[2], void* C,
+                          int64_t ldc, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  using namespace b2;
+  if (!is_op(transa)) return -1;
+  if (!is_op(transb)) return -2;
+  if (!alpha) return -6;
+  if (!beta) return -11;
+  const double ar = alpha[0], ai = alpha[1], br = beta[0], bi = beta[1];
+  const bool alpha0 = (ar == 0.0 && ai == 0.0);
+  const bool scale_only = alpha0 || k == 0;
+  const int bad = check_gemm_args(transa, transb, m, n, k, A, lda, B, ldb, C, ldc, !scale_only);
+  if (bad) return bad;
+  if (m == 0 || n == 0) return B2_OK;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  double2* Cz = static_cast<double2*>(C);
+  if (scale_only) {
+    if (br == 1.0 && bi == 0.0) return B2_OK;
+    zscale_kernel<<<grid_for(m * n), 256, 0, st>>>(m, n, br, bi, Cz, ldc);
+    return cudaGetLastError() == cudaSuccess ? B2_OK : B2_ERR_LAUNCH;
+  }
+  const Plan p = make_plan(transa, transb, m, n, k);
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) != 0 ||
+      workspace_bytes < 3 * (p.sa + p.sb + p.sc))
+    return B2_ERR_WORKSPACE;
+  char* w = static_cast<char*>(workspace);
+  double* Ap[3];
+  double* Bp[3];
+  double* T[3];
+  for (int i = 0; i < 3; ++i) {
+    Ap[i] = reinterpret_cast<double*>(w + i * p.sa);
+    Bp[i] = reinterpret_cast<double*>(w + 3 * p.sa + i * p.sb);
+    T[i] = reinterpret_cast<double*>(w + 3 * p.sa + 3 * p.sb + i * p.sc);
+  }
+  zsplit_scale_kernel<<<grid_for(p.ra * p.ca), 256, 0, st>>>(p.ra, p.ca, static_cast<const double2*>(A), lda, ar, ai,
+                                                           is_c(transa), Ap[0], Ap[1], Ap[2], p.lpa);
+  zsplit_scale_kernel<<<grid_for(p.rb * p.cb), 256, 0, st>>>(p.rb, p.cb, static_cast<const double2*>(B), ldb, 1.0,
+                                                           0.0, is_c(transb), Bp[0], Bp[1], Bp[2], p.lpb);
+  if (cudaGetLastError() != cudaSuccess) return B2_ERR_LAUNCH;
+  const char ta = real_op(transa), tb = real_op(transb);
+  for (int i = 0; i < 3; ++i) {  // T1 = A'r*Br, T2 = A'i*Bi, T3 = (A'r+A'i)*(Br+Bi)
+    const int rc = gemm_entry<double>(B2_VARIANT_AUTO, ta, tb, m, n, k, 1.0, Ap[i], p.lpa, Bp[i], p.lpb, 0.0, T[i],
+                                      p.lpc, st);
+    if (rc) return rc;
+  }
+  zmerge3m_kernel<<<grid_for(m * n), 256, 0, st>>>(m, n, T[0], T[1], T[2], p.lpc, br, bi, Cz, ldc);
+  return cudaGetLastError() == cudaSuccess ? B2_OK : B2_ERR_LAUNCH;
+}
+
 // ---- b2_zgemm4m without a caller-provided workspace -------------------------------------------
 // The scratch planes live in the library image.  In host code the array's name is only a
 // host-side stand-in for the symbol, not a device address: the address each device maps it
@@ -166,7 +256,7 @@ extern "C" int b2_zgemm4m_static(char transa, char transb, int64_t m, int64_t n,
                                  void* C, int64_t ldc, void* cuda_stream) {
   using namespace b2;
   static void* scratch_by_device[64] = {};
-  if ((is_n(transa) || is_t(transa)) && (is_n(transb) || is_t(transb)) && m >= 0 && n >= 0 && k >= 0 &&
+  if (is_op(transa) && is_op(transb) && m >= 0 && n >= 0 && k >= 0 &&
       make_plan(transa, transb, m, n, k).total > (size_t)B2_ZGEMM4M_STATIC_BYTES)
     return B2_ERR_STATIC_LIMIT;
   int dev = -1;

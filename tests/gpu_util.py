@@ -8,7 +8,7 @@ import torch
 from helpers import U
 from paper_1611_08035_b200 import synth
 
-TORCH_DT = {"d": torch.float64, "s": torch.float32, "z": torch.complex128}
+TORCH_DT = {"d": torch.float64, "s": torch.float32, "z": torch.complex128, "z3": torch.complex128}
 
 
 def sample_columns(n: int, tile: int = 64, extra: int = 24, seed: int = 0):
@@ -23,9 +23,9 @@ def sample_columns(n: int, tile: int = 64, extra: int = 24, seed: int = 0):
 
 def run_and_check(b2, oracle, kind, transa, transb, m, n, k, alpha, beta, dist="uniform", seed=0, pad=False,
                   variant=None, cols=None, c_dist=None, expect_exact=False, lds=None, offset=0, factor=None):
-    """Returns the largest observed error/bound ratio.  kind: 'd', 's' (real) or 'z' (4M complex).
+    """Returns the largest observed error/bound ratio.  kind: 'd', 's' (real), 'z' (4M complex) or 'z3' (3M).
 
-    Checks: every compared element within 2*k*u*S (complex: 2*(2k+4)*u*S per component); bit-exact when
+    Checks: every compared element within 2*k*u*S (complex: 2*(2k+4)*u*S per component, 3M 2*(3k+6)*u*S); bit-exact when
     expect_exact; padding rows of C and unsampled nothing-else untouched; A and B unchanged.
     `offset` shifts every base pointer by that many elements (misaligned bases)."""
     tdt = TORCH_DT[kind]
@@ -54,6 +54,10 @@ def run_and_check(b2, oracle, kind, transa, transb, m, n, k, alpha, beta, dist="
         ws = torch.empty(max(256, b2.b2_zgemm4m_workspace_bytes(transa, transb, m, n, k)), dtype=torch.uint8,
                          device="cuda")
         b2.b2_zgemm4m(transa, transb, m, n, k, alpha, Ad, lda, Bd, ldb, beta, Cd, ldc, ws)
+    elif kind == "z3":
+        ws = torch.empty(max(256, b2.b2_zgemm3m_workspace_bytes(transa, transb, m, n, k)), dtype=torch.uint8,
+                         device="cuda")
+        b2.b2_zgemm3m(transa, transb, m, n, k, alpha, Ad, lda, Bd, ldb, beta, Cd, ldc, ws)
     else:
         fn = b2.b2_dgemm if kind == "d" else b2.b2_sgemm
         rc = fn(transa, transb, m, n, k, alpha, Ad, lda, Bd, ldb, beta, Cd, ldc, variant=variant, check=False)
@@ -90,13 +94,13 @@ def run_and_check(b2, oracle, kind, transa, transb, m, n, k, alpha, beta, dist="
         assert g.tobytes() == w.tobytes(), "integer-valued problem is not bit-exact"
         return 0.0
     u = U[np.dtype(Cn.dtype)]
-    if kind == "z":
-        bound = 2.0 * (2 * k + 4) * u * Sv
+    if kind in ("z", "z3"):
+        bound = 2.0 * ((2 * k + 4) if kind == "z" else (3 * k + 6)) * u * Sv
         err = np.maximum(np.abs(g.real - w.real), np.abs(g.imag - w.imag))
     else:
         bound = (2.0 * k * u if factor is None else factor) * Sv
         err = np.abs(g.astype(np.float64) - w.astype(np.float64))
-    assert np.all(np.isfinite(g.view(np.float64) if kind == "z" else g)), "non-finite result"
+    assert np.all(np.isfinite(g.view(np.float64) if kind in ("z", "z3") else g)), "non-finite result"
     bad = err > bound
     assert not bad.any(), f"{int(bad.sum())} elements exceed the bound; worst ratio " \
                           f"{float((err / np.maximum(bound, 1e-300)).max()):.3g}"

@@ -58,7 +58,7 @@ def test_argument_checks_need_no_gpu(b2):
     assert dgemm(b"N", b"N", 2, 0, 2, 2, 2, 2, A=None, B=None, C=None) == 0
     assert lib.b2_dgemm_variant(77, b"N", b"N", 2, 2, 2, d(1.0), fake, 2, fake, 2, d(0.0), fake, 2, None) == 1004
     al = (d * 2)(1.0, 0.0)
-    assert lib.b2_zgemm4m(b"C", b"N", 2, 2, 2, al, fake, 2, fake, 2, al, fake, 2, fake, 0, None) == -1
+    assert lib.b2_zgemm4m(b"X", b"N", 2, 2, 2, al, fake, 2, fake, 2, al, fake, 2, fake, 0, None) == -1
     assert lib.b2_zgemm4m(b"N", b"N", 2, 2, 2, None, fake, 2, fake, 2, al, fake, 2, fake, 0, None) == -6
     assert lib.b2_zgemm4m(b"N", b"N", 2, 2, 2, al, fake, 2, fake, 2, None, fake, 2, fake, 0, None) == -11
     assert lib.b2_zgemm4m(b"N", b"N", 2, 2, 2, al, fake, 1, fake, 2, al, fake, 2, fake, 0, None) == -8
@@ -73,7 +73,9 @@ def test_argument_checks_need_no_gpu(b2):
 def test_workspace_sizes(b2):
     assert b2.b2_zgemm4m_workspace_bytes("N", "N", 4096, 4096, 4096) == 6 * 4096 * 4096 * 8
     assert b2.b2_zgemm4m_workspace_bytes("N", "N", 3, 5, 7) % 256 == 0
-    assert b2.b2_zgemm4m_workspace_bytes("C", "N", 3, 5, 7) == 0
+    assert b2.b2_zgemm4m_workspace_bytes("X", "N", 3, 5, 7) == 0
+    assert b2.b2_zgemm4m_workspace_bytes("C", "N", 3, 5, 7) == b2.b2_zgemm4m_workspace_bytes("T", "N", 3, 5, 7)
+    assert b2.b2_zgemm3m_workspace_bytes("N", "N", 4096, 4096, 4096) == 9 * 4096 * 4096 * 8
     assert b2.b2_gemm_host_workspace_bytes(0, "N", "N", 8192, 8192, 8192) == 3 * 8192 * 8192 * 8
     assert b2.b2_gemm_host_workspace_bytes(1, "T", "N", 1001, 999, 1003) >= 4 * (1003 * 1001 + 1003 * 999 + 1001 * 999)
 

@@ -270,11 +270,32 @@ def test_zgemm4m_small_full_all_transposes(b2, oracle):
     run_and_check(b2, oracle, "z", "N", "N", 0, 17, 9, 1 + 0j, 0j, seed=56)
 
 
+def test_zgemm_conjugate_transposes_and_3m(b2, oracle):
+    """Every op pair with a conjugate transpose through 4M, and all nine pairs through 3M: integer data bit-exact
+    against direct complex arithmetic, uniform data within 2*(2k+4)*u*S (4M) / 2*(3k+6)*u*S (3M) per component."""
+    for ta in "NTC":
+        for tb in "NTC":
+            for kind in ("z", "z3"):
+                if kind == "z" and "C" not in (ta, tb):
+                    continue  # covered by test_zgemm4m_small_full_all_transposes
+                run_and_check(b2, oracle, kind, ta, tb, 301, 203, 157, 1 + 0.5j, 0j, seed=61, pad=True)
+                run_and_check(b2, oracle, kind, ta, tb, 130, 70, 33, 0.3 - 0.8j, 0.25 + 0.75j, seed=62, pad=True)
+                run_and_check(b2, oracle, kind, ta, tb, 130, 70, 33, 2 - 1j, 0.5 + 0.5j, dist="int9", seed=63,
+                              expect_exact=True)
+    run_and_check(b2, oracle, "z3", "N", "N", 33, 17, 0, 1 + 1j, 0.5 - 0.5j, seed=64)
+    run_and_check(b2, oracle, "z3", "C", "N", 33, 17, 5, 0j, 0.5 - 0.5j, seed=65)
+
+
+def test_zgemm3m_4096_sampled(b2, oracle):
+    cols = sample_columns(4096, tile=64, extra=8, seed=6)
+    run_and_check(b2, oracle, "z3", "N", "N", 4096, 4096, 4096, 1 + 0.5j, 0j, dist="uniform", seed=5000, cols=cols)
+
+
 def test_zgemm4m_argument_errors(b2):
     z = torch.zeros(64, dtype=torch.complex128, device="cuda")
     ws = torch.empty(1 << 16, dtype=torch.uint8, device="cuda")
-    assert b2.b2_zgemm4m("C", "N", 4, 4, 4, 1, z, 4, z, 4, 0, z, 4, ws, check=False) == -1
-    assert b2.b2_zgemm4m("N", "C", 4, 4, 4, 1, z, 4, z, 4, 0, z, 4, ws, check=False) == -2
+    assert b2.b2_zgemm4m("X", "N", 4, 4, 4, 1, z, 4, z, 4, 0, z, 4, ws, check=False) == -1
+    assert b2.b2_zgemm4m("N", "H", 4, 4, 4, 1, z, 4, z, 4, 0, z, 4, ws, check=False) == -2
     assert b2.b2_zgemm4m("N", "N", 4, 4, 4, 1, z, 4, z, 4, 0, z, 4, None, check=False) == 1003
     assert b2.b2_zgemm4m("N", "N", 4, 4, 4, 1, z, 4, z, 4, 0, z, 4, ws[:64], check=False) == 1003
     assert b2.b2_zgemm4m("N", "N", 4, 4, 4, 1, z, 4, z, 4, 0, z, 4, ws[8:], check=False) == 1003  # misaligned
