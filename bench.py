@@ -215,6 +215,20 @@ def other_configs(b2, device):
     g = quick_gflops(lambda: b2.b2_zgemm4m("N", "N", m, n, k, 1 + 0.5j, A, m, B, k, 0j, C, m, ws), 8.0 * m * n * k,
                      iters=2, warm=2)
     out.append({"workload": "zgemm4m_nn_4096", "gflops": round(g, 1), "frac_of_peak": round(g / 1e3 / FP64_PEAK_TFLOPS, 4)})
+    # small m*n, long k: split-K against the plain kernel
+    sm, sn, sk = 256, 256, 65536
+    As = synth.matrix(sm, sk, sm, "uniform", 71, torch.float64, device=device)
+    Bs = synth.matrix(sk, sn, sk, "uniform", 72, torch.float64, device=device)
+    Cs = torch.zeros(sm * sn, dtype=torch.float64, device=device)
+    wss = torch.empty(max(256, b2.b2_gemm_splitk_workspace_bytes(torch.float64, sm, sn, sk, 0)), dtype=torch.uint8,
+                      device=device)
+    g0 = quick_gflops(lambda: b2.b2_dgemm("N", "N", sm, sn, sk, 1.0, As, sm, Bs, sk, 0.0, Cs, sm), 2.0 * sm * sn * sk,
+                      iters=5, warm=2)
+    g1 = quick_gflops(lambda: b2.b2_gemm_splitk("N", "N", sm, sn, sk, 1.0, As, sm, Bs, sk, 0.0, Cs, sm, 0, wss),
+                      2.0 * sm * sn * sk, iters=5, warm=2)
+    out.append({"workload": "dgemm_splitk_256x256x65536", "gflops": round(g1, 1), "plain_kernel_gflops": round(g0, 1),
+                "splits": b2.b2_gemm_splitk_auto(sm, sn, sk), "frac_of_peak": round(g1 / 1e3 / FP64_PEAK_TFLOPS, 4)})
+    del As, Bs, Cs, wss
     del ws
     ws = torch.empty(b2.b2_zgemm3m_workspace_bytes("N", "N", m, n, k), dtype=torch.uint8, device=device)
     g = quick_gflops(lambda: b2.b2_zgemm3m("N", "N", m, n, k, 1 + 0.5j, A, m, B, k, 0j, C, m, ws), 8.0 * m * n * k,

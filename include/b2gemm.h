@@ -204,6 +204,31 @@ int b2_sgemm_strided_batched(char transa, char transb, int64_t m, int64_t n, int
                              float* C, int64_t ldc, int64_t stride_c, int64_t batch, void* cuda_stream);
 
 /*
+ * Split-K GEMM for small m*n with long k.  One CTA per C tile leaves most SMs idle when m*n is small, however
+ * long k is; here k is cut into `splits` contiguous chunks (whole 16-deep slabs), the chunks' partial products
+ * are computed by one batched launch of the GEMM kernel into workspace planes, and a second kernel stores
+ * C = alpha*(P_0 + P_1 + ... ) + beta*C with the planes added in ascending chunk order.  The result therefore
+ * does not depend on scheduling (same bits on every run); it is the plain GEMM definition with a different,
+ * fixed summation order (the paper, Section 2.1, fixes no order), so the b2_dgemm error bound applies and
+ * integer-valued problems are bit-exact.
+ *   splits     0 = chosen by the library (b2_gemm_splitk_auto: as many chunks as it takes to fill the SMs with
+ *              64 x 64 tiles, each chunk at least 256 deep, at most 64); 1 = plain b2_dgemm; > k is cut to k.
+ *   workspace  DEVICE memory, 256-byte aligned, at least b2_gemm_splitk_workspace_bytes(dtype, m, n, k, splits)
+ *              bytes (dtype 0 = fp64, 1 = fp32; 0 bytes when the call degenerates to the plain GEMM);
+ *              owned by the caller, overwritten.
+ * Other arguments, quick returns and error numbering as b2_dgemm; splits < 0 returns -14; a missing, misaligned or
+ * short workspace returns B2_ERR_WORKSPACE and launches nothing.
+ */
+int b2_gemm_splitk_auto(int64_t m, int64_t n, int64_t k);
+size_t b2_gemm_splitk_workspace_bytes(int dtype, int64_t m, int64_t n, int64_t k, int splits);
+int b2_dgemm_splitk(char transa, char transb, int64_t m, int64_t n, int64_t k, double alpha, const double* A,
+                    int64_t lda, const double* B, int64_t ldb, double beta, double* C, int64_t ldc, int splits,
+                    void* workspace, size_t workspace_bytes, void* cuda_stream);
+int b2_sgemm_splitk(char transa, char transb, int64_t m, int64_t n, int64_t k, float alpha, const float* A,
+                    int64_t lda, const float* B, int64_t ldb, float beta, float* C, int64_t ldc, int splits,
+                    void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
  * fp32 GEMM on the tensor cores in TF32 -- separate entry points because TF32 changes results (b2_sgemm
  * never uses it).  The paper has no counterpart; the operation is the same BLAS GEMM with the products taken
  * in the TF32 format (1 sign, 8 exponent, 10 mantissa bits) and accumulated in fp32:

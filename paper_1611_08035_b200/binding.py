@@ -36,6 +36,12 @@ _SIGNATURES = {
     "b2_zgemm4m": (c_int, [c_char, c_char, c_int64, c_int64, c_int64, ctypes.POINTER(c_double), c_void_p, c_int64,
                            c_void_p, c_int64, ctypes.POINTER(c_double), c_void_p, c_int64, c_void_p, c_size_t,
                            c_void_p]),
+    "b2_gemm_splitk_auto": (c_int, [c_int64, c_int64, c_int64]),
+    "b2_gemm_splitk_workspace_bytes": (c_size_t, [c_int, c_int64, c_int64, c_int64, c_int]),
+    "b2_dgemm_splitk": (c_int, [c_char, c_char, c_int64, c_int64, c_int64, c_double, c_void_p, c_int64, c_void_p, c_int64,
+                                c_double, c_void_p, c_int64, c_int, c_void_p, c_size_t, c_void_p]),
+    "b2_sgemm_splitk": (c_int, [c_char, c_char, c_int64, c_int64, c_int64, c_float, c_void_p, c_int64, c_void_p, c_int64,
+                                c_float, c_void_p, c_int64, c_int, c_void_p, c_size_t, c_void_p]),
     "b2_zgemm3m_workspace_bytes": (c_size_t, [c_char, c_char, c_int64, c_int64, c_int64]),
     "b2_zgemm3m": (c_int, [c_char, c_char, c_int64, c_int64, c_int64, ctypes.POINTER(c_double), c_void_p, c_int64,
                            c_void_p, c_int64, ctypes.POINTER(c_double), c_void_p, c_int64, c_void_p, c_size_t,
@@ -182,6 +188,35 @@ def b2_zgemm4m(transa, transb, m, n, k, alpha, A, lda, B, ldb, beta, C, ldc, wor
                           _ptr(workspace), wbytes, _stream())
     if check:
         _check("b2_zgemm4m", rc)
+    return rc
+
+
+def b2_gemm_splitk_auto(m, n, k) -> int:
+    return lib().b2_gemm_splitk_auto(m, n, k)
+
+
+def b2_gemm_splitk_workspace_bytes(dtype, m, n, k, splits=0) -> int:
+    """dtype: torch.float64 / torch.float32."""
+    return lib().b2_gemm_splitk_workspace_bytes(0 if dtype == torch.float64 else 1, m, n, k, splits)
+
+
+def b2_gemm_splitk(transa, transb, m, n, k, alpha, A, lda, B, ldb, beta, C, ldc, splits=0, workspace=None,
+                   check=True) -> int:
+    """Split-K GEMM (fp64 or fp32 by the tensors' dtype); workspace: uint8 CUDA tensor or None."""
+    if C.dtype == torch.float64:
+        fn, name = lib().b2_dgemm_splitk, "b2_dgemm_splitk"
+    elif C.dtype == torch.float32:
+        fn, name = lib().b2_sgemm_splitk, "b2_sgemm_splitk"
+    else:
+        raise TypeError("b2_gemm_splitk takes float64 or float32 tensors")
+    for t in (A, B, C):
+        if t is not None and (t.dtype != C.dtype or not t.is_cuda):
+            raise TypeError("b2_gemm_splitk takes CUDA tensors of one dtype")
+    wbytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    rc = fn(_tr(transa), _tr(transb), m, n, k, alpha, _ptr(A), lda, _ptr(B), ldb, beta, _ptr(C), ldc, splits,
+            _ptr(workspace), wbytes, _stream())
+    if check:
+        _check(name, rc)
     return rc
 
 

@@ -121,7 +121,7 @@ static bool operands_aligned(const T* A, int64_t lda, const T* B, int64_t ldb) {
 
 // `aligned`: A and B have 16-byte aligned columns, which the TMA-staged variants need.
 template <typename T>
-int choose_variant(int64_t m, int64_t n, int64_t k, bool aligned) {
+int choose_variant(int64_t m, int64_t n, int64_t k, bool aligned, int64_t batch = 1) {
   const int count = variant_count_t<T>();
   TileChoice cand[16];
   for (int v = 0; v < count && v < 16; ++v) {
@@ -131,7 +131,7 @@ int choose_variant(int64_t m, int64_t n, int64_t k, bool aligned) {
     cand[v] = TileChoice{vi.bm, vi.bn, vi.bk, vi.threads, vi.ctas_per_sm, vi.efficiency,
                          comparison_only || (needs_alignment && !aligned)};
   }
-  return select_tile(cand, count < 16 ? count : 16, m, n, k, sm_count_cached(), (int)sizeof(T));
+  return select_tile(cand, count < 16 ? count : 16, m, n, k, sm_count_cached(), (int)sizeof(T), batch);
 }
 
 // Variant choice and launch of an already checked, non-trivial problem (m, n, k > 0, alpha != 0).
@@ -144,7 +144,7 @@ int gemm_launch_checked(int variant, bool ta, bool tb, int64_t m, int64_t n, int
   constexpr int64_t kVec = 16 / (int64_t)sizeof(T);
   const bool aligned = operands_aligned(A, lda, B, ldb) &&
                        (ex.batch <= 1 || (ex.stride_a % kVec == 0 && ex.stride_b % kVec == 0));
-  if (variant == B2_VARIANT_AUTO) variant = choose_variant<T>(m, n, k, aligned && ex.batch <= 1);
+  if (variant == B2_VARIANT_AUTO) variant = choose_variant<T>(m, n, k, aligned && ex.batch <= 1, ex.batch);
   GemmArgs<T> args;
   args.m = m, args.n = n, args.k = k;
   args.alpha = alpha, args.beta = beta;

@@ -1,6 +1,7 @@
 // Level-3 routines built on the GEMM kernel (the paper's Abstract and Introduction name the level-3 BLAS as
 // its consumers): the symmetric rank-k update, which is a GEMM with op(B) = op(A)^T restricted to one triangle of
-// C, and the strided-batched GEMM, which is the GEMM grid replicated along grid.y.
+// C, the strided-batched GEMM, which is the GEMM grid replicated along grid.y, and a split-K GEMM for small
+// m*n with long k, which is a batched GEMM over k-chunks followed by an ordered sum.
 #include "b2gemm.h"
 #include "entry.h"
 
@@ -115,6 +116,91 @@ int gemm_strided_batched(char transa, char transb, int64_t m, int64_t n, int64_t
   return B2_OK;
 }
 
+// ---- split-K: k cut into contiguous chunks, one partial product per chunk, summed in a fixed order ---------
+// For small m*n and large k one CTA per C tile leaves most SMs idle; the chunks run as the batch dimension of
+// one launch (A and B advance by one chunk per batch index, partial products go to workspace planes) and a
+// second kernel forms C = alpha*(P_0 + P_1 + ...) + beta*C with the planes added in ascending order, so the
+// result does not depend on scheduling.
+template <typename T>
+__global__ void splitk_reduce_kernel(int64_t m, int64_t n, int planes, const T* __restrict__ P, int64_t ldp,
+                                     int64_t plane_stride, T alpha, T beta, T* __restrict__ C, int64_t ldc) {
+  const int64_t total = m * n;
+  for (int64_t idx = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; idx < total;
+       idx += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t r = idx % m, c = idx / m;
+    const T* p = P + r + c * ldp;
+    T acc = p[0];
+    for (int s = 1; s < planes; ++s) acc += p[s * plane_stride];
+    T* dst = C + r + c * ldc;
+    *dst = (beta == T(0)) ? alpha * acc : alpha * acc + beta * *dst;
+  }
+}
+
+constexpr int kSplitChunkUnit = 16;  // chunks are whole k-slabs, which also keeps every chunk 16-byte aligned
+
+template <typename T>
+int64_t splitk_pitch(int64_t m) {
+  const int64_t vec = 16 / (int64_t)sizeof(T);
+  return m < 1 ? vec : (m + vec - 1) / vec * vec;
+}
+
+int splitk_auto(int64_t m, int64_t n, int64_t k) {
+  if (m <= 0 || n <= 0 || k <= 0) return 1;
+  const int64_t tiles = ((m + 63) / 64) * ((n + 63) / 64);
+  const int64_t slots = 148 * 4;  // resident 64 x 64 tiles
+  int64_t s = slots / tiles;
+  if (s > k / 256) s = k / 256;  // every chunk at least 256 deep
+  if (s > 64) s = 64;
+  return s < 1 ? 1 : (int)s;
+}
+
+template <typename T>
+int gemm_splitk(char transa, char transb, int64_t m, int64_t n, int64_t k, T alpha, const T* A, int64_t lda,
+                const T* B, int64_t ldb, T beta, T* C, int64_t ldc, int splits, void* workspace,
+                size_t workspace_bytes, void* cuda_stream) {
+  const bool scale_only = (alpha == T(0) || k == 0);
+  const int bad = check_gemm_args(transa, transb, m, n, k, A, lda, B, ldb, C, ldc, !scale_only);
+  if (bad) return bad;
+  if (splits < 0) return -14;
+  if (splits == 0) splits = splitk_auto(m, n, k);
+  if (splits > k) splits = k > 0 ? (int)k : 1;
+  if (scale_only || splits <= 1 || m == 0 || n == 0)
+    return gemm_entry<T>(B2_VARIANT_AUTO, transa, transb, m, n, k, alpha, A, lda, B, ldb, beta, C, ldc, cuda_stream);
+  const int64_t chunk = ((k + splits - 1) / splits + kSplitChunkUnit - 1) / kSplitChunkUnit * kSplitChunkUnit;
+  const int64_t full = k / chunk, rest = k - full * chunk;
+  const int planes = (int)(full + (rest > 0 ? 1 : 0));
+  const int64_t ldp = splitk_pitch<T>(m), plane_stride = ldp * n;
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) != 0 ||
+      workspace_bytes < (size_t)planes * (size_t)plane_stride * sizeof(T))
+    return B2_ERR_WORKSPACE;
+  T* P = static_cast<T*>(workspace);
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  const bool ta = l3_is_t(transa), tb = l3_is_t(transb);
+  const int64_t step_a = ta ? chunk : chunk * lda, step_b = tb ? chunk * ldb : chunk;  // one chunk further along k
+  if (full > 0) {
+    GemmExtra ex;
+    ex.batch = (int)full, ex.stride_a = step_a, ex.stride_b = step_b, ex.stride_c = plane_stride;
+    const int rc = gemm_launch_checked<T>(B2_VARIANT_AUTO, ta, tb, m, n, chunk, T(1), A, lda, B, ldb, T(0), P, ldp, ex, st);
+    if (rc) return rc;
+  }
+  if (rest > 0) {
+    const int rc = gemm_launch_checked<T>(B2_VARIANT_AUTO, ta, tb, m, n, rest, T(1), A + full * step_a, lda,
+                                          B + full * step_b, ldb, T(0), P + full * plane_stride, ldp, GemmExtra(), st);
+    if (rc) return rc;
+  }
+  splitk_reduce_kernel<T><<<blocks_for(m * n), 256, 0, st>>>(m, n, planes, P, ldp, plane_stride, alpha, beta, C, ldc);
+  return cudaGetLastError() == cudaSuccess ? B2_OK : B2_ERR_LAUNCH;
+}
+
+template <typename T>
+size_t splitk_workspace_bytes(int64_t m, int64_t n, int64_t k, int splits) {
+  if (m <= 0 || n <= 0 || k <= 0 || splits < 0) return 0;
+  if (splits == 0) splits = splitk_auto(m, n, k);
+  if (splits > k) splits = (int)k;
+  if (splits <= 1) return 0;
+  return (size_t)splits * (size_t)splitk_pitch<T>(m) * (size_t)n * sizeof(T);
+}
+
 }  // namespace
 }  // namespace b2
 
@@ -139,4 +225,22 @@ extern "C" int b2_sgemm_strided_batched(char transa, char transb, int64_t m, int
                                         int64_t batch, void* cuda_stream) {
   return b2::gemm_strided_batched<float>(transa, transb, m, n, k, alpha, A, lda, stride_a, B, ldb, stride_b, beta, C,
                                          ldc, stride_c, batch, cuda_stream);
+}
+
+extern "C" int b2_gemm_splitk_auto(int64_t m, int64_t n, int64_t k) { return b2::splitk_auto(m, n, k); }
+extern "C" size_t b2_gemm_splitk_workspace_bytes(int dtype, int64_t m, int64_t n, int64_t k, int splits) {
+  return dtype == 0 ? b2::splitk_workspace_bytes<double>(m, n, k, splits)
+                    : b2::splitk_workspace_bytes<float>(m, n, k, splits);
+}
+extern "C" int b2_dgemm_splitk(char transa, char transb, int64_t m, int64_t n, int64_t k, double alpha, const double* A,
+                               int64_t lda, const double* B, int64_t ldb, double beta, double* C, int64_t ldc,
+                               int splits, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  return b2::gemm_splitk<double>(transa, transb, m, n, k, alpha, A, lda, B, ldb, beta, C, ldc, splits, workspace,
+                                 workspace_bytes, cuda_stream);
+}
+extern "C" int b2_sgemm_splitk(char transa, char transb, int64_t m, int64_t n, int64_t k, float alpha, const float* A,
+                               int64_t lda, const float* B, int64_t ldb, float beta, float* C, int64_t ldc, int splits,
+                               void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  return b2::gemm_splitk<float>(transa, transb, m, n, k, alpha, A, lda, B, ldb, beta, C, ldc, splits, workspace,
+                                workspace_bytes, cuda_stream);
 }

@@ -38,9 +38,11 @@ inline MachineRates machine_rates(int elem_bytes) {
 }
 
 // Estimated clocks for one SM to finish its share of the problem with tile `c`.
-inline double estimate_clks(const TileChoice& c, int64_t m, int64_t n, int64_t k, int sms, int elem_bytes) {
+// `batch` independent problems of this shape share one launch (their tiles fill the SMs together).
+inline double estimate_clks(const TileChoice& c, int64_t m, int64_t n, int64_t k, int sms, int elem_bytes,
+                            int64_t batch = 1) {
   const MachineRates r = machine_rates(elem_bytes);
-  const double tiles = (double)((m + c.bm - 1) / c.bm) * (double)((n + c.bn - 1) / c.bn);
+  const double tiles = (double)((m + c.bm - 1) / c.bm) * (double)((n + c.bn - 1) / c.bn) * (double)(batch < 1 ? 1 : batch);
   const double kt = (double)((k + c.bk - 1) / c.bk);
   // tiles are handed out CTA by CTA; an SM ends up with ceil(tiles / sms) of them
   const double per_sm = (double)(int64_t)((tiles + sms - 1) / sms);
@@ -65,12 +67,13 @@ inline double estimate_clks(const TileChoice& c, int64_t m, int64_t n, int64_t k
 }
 
 // Index of the candidate with the smallest estimate.
-inline int select_tile(const TileChoice* cand, int count, int64_t m, int64_t n, int64_t k, int sms, int elem_bytes) {
+inline int select_tile(const TileChoice* cand, int count, int64_t m, int64_t n, int64_t k, int sms, int elem_bytes,
+                       int64_t batch = 1) {
   int best = -1;
   double best_t = 0.0;
   for (int i = 0; i < count; ++i) {
     if (cand[i].explicit_only) continue;
-    const double t = estimate_clks(cand[i], m, n, k, sms, elem_bytes);
+    const double t = estimate_clks(cand[i], m, n, k, sms, elem_bytes, batch);
     if (best < 0 || t < best_t) best = i, best_t = t;
   }
   return best < 0 ? 0 : best;

@@ -112,3 +112,68 @@ def test_strided_batched(b2, oracle, kind):
     assert b2.b2_gemm_strided_batched("N", "N", 4, 4, 4, 1.0, z, 4, -1, z, 4, 16, 0.0, z, 4, 16, 2, check=False) == -9
     assert b2.b2_gemm_strided_batched("N", "N", 4, 4, 4, 1.0, z, 4, 16, z, 4, 16, 0.0, z, 4, 16, -1, check=False) == -17
     assert b2.b2_gemm_strided_batched("N", "N", 4, 4, 4, 1.0, z, 4, 16, z, 4, 16, 0.0, z, 4, 16, 0) == 0
+
+
+# ---- split-K -------------------------------------------------------------------------------------------
+
+def run_splitk(b2, oracle, kind, ta, tb, m, n, k, alpha, beta, splits, dist="uniform", seed=0, pad=False, exact=False):
+    """The oracle is the plain GEMM definition: split-K only fixes another summation order."""
+    tdt, ndt = DT[kind]
+    (ra, _), (rb, _) = synth.operand_shapes(ta, tb, m, n, k)
+    lds = (synth.padded_ld(ra), synth.padded_ld(rb), synth.padded_ld(m)) if pad else (None, None, None)
+    A, lda, B, ldb, C, ldc = synth.gemm_inputs(ta, tb, m, n, k, dist, seed, tdt, *lds)
+    want = C.numpy().copy()
+    oracle.ref_gemm(ta, tb, m, n, k, alpha, A.numpy(), lda, B.numpy(), ldb, beta, want, ldc)
+    need = b2.b2_gemm_splitk_workspace_bytes(tdt, m, n, k, splits)
+    ws = torch.empty(max(256, need), dtype=torch.uint8, device="cuda")
+    outs = []
+    for _ in range(2):
+        Cd = C.cuda()
+        b2.b2_gemm_splitk(ta, tb, m, n, k, alpha, A.cuda(), lda, B.cuda(), ldb, beta, Cd, ldc, splits, ws)
+        assert b2.b2_device_status() == 0
+        outs.append(Cd.cpu().numpy())
+    assert outs[0].tobytes() == outs[1].tobytes(), "two runs differ"
+    got = outs[0]
+    if m == 0 or n == 0:
+        assert got.tobytes() == C.numpy().tobytes()
+        return
+    G, W, C0 = (x.reshape(n, ldc) for x in (got, want, C.numpy()))
+    assert G[:, m:].tobytes() == C0[:, m:].tobytes(), "padding rows of C were written"
+    if exact:
+        assert G[:, :m].tobytes() == W[:, :m].tobytes()
+        return
+    _, S = oracle.ref_gemm_hi(ta, tb, m, n, k, alpha, A.numpy(), lda, B.numpy(), ldb, beta, C.numpy(), ldc)
+    err = np.abs(G[:, :m].astype(np.float64) - W[:, :m].astype(np.float64))
+    assert np.all(err <= 2 * max(k, 1) * U[np.dtype(ndt)] * S.reshape(n, max(1, m))[:, :m])
+
+
+@pytest.mark.parametrize("kind", ["d", "s"])
+def test_splitk_matches_the_plain_definition(b2, oracle, kind):
+    for ta, tb in itertools.product("NT", "NT"):
+        run_splitk(b2, oracle, kind, ta, tb, 100, 70, 2000, 0.7, -0.3, splits=0, seed=1, pad=True)
+        run_splitk(b2, oracle, kind, ta, tb, 64, 64, 4096, 1.5, 0.5, splits=7, dist="int9", seed=2, exact=True)
+        run_splitk(b2, oracle, kind, ta, tb, 130, 33, 1000, 1.0, 0.0, splits=5, seed=3)          # ragged last chunk
+    for (m, n, k, splits) in [(1, 1, 5000, 0), (17, 9, 31, 4), (17, 9, 31, 40), (50, 60, 16, 3), (8, 8, 0, 4),
+                              (0, 5, 100, 2), (33, 65, 257, 1), (256, 256, 8192, 0)]:
+        run_splitk(b2, oracle, kind, "N", "N", m, n, k, -1.0, 1.0, splits=splits, dist="int9", seed=m + k, exact=True)
+
+
+def test_splitk_plan_and_workspace_errors(b2):
+    assert b2.b2_gemm_splitk_auto(256, 256, 65536) == 37   # 16 tiles of 64 x 64 on 592 resident slots
+    assert b2.b2_gemm_splitk_auto(8192, 8192, 8192) == 1
+    assert b2.b2_gemm_splitk_auto(64, 64, 1024) == 4       # chunks stay at least 256 deep
+    assert b2.b2_gemm_splitk_workspace_bytes(torch.float64, 100, 10, 4096, 4) == 4 * 100 * 10 * 8
+    assert b2.b2_gemm_splitk_workspace_bytes(torch.float32, 5, 10, 4096, 4) == 4 * 8 * 10 * 4
+    assert b2.b2_gemm_splitk_workspace_bytes(torch.float64, 100, 10, 4096, 1) == 0
+    A = torch.ones(64 * 1024, dtype=torch.float64, device="cuda")
+    C = torch.zeros(64 * 64, dtype=torch.float64, device="cuda")
+    ws = torch.empty(4 * 64 * 64 * 8, dtype=torch.uint8, device="cuda")
+    args = ("N", "N", 64, 64, 1024, 1.0, A, 64, A, 1024, 0.0, C, 64)
+    assert b2.b2_gemm_splitk(*args, splits=-1, workspace=ws, check=False) == -14
+    assert b2.b2_gemm_splitk(*args, splits=4, workspace=None, check=False) == 1003
+    assert b2.b2_gemm_splitk(*args, splits=4, workspace=ws[:1000], check=False) == 1003
+    torch.cuda.synchronize()
+    assert (C == 0).all()
+    assert b2.b2_gemm_splitk(*args, splits=4, workspace=ws) == 0
+    torch.cuda.synchronize()
+    assert (C == 1024).all()
