@@ -49,6 +49,11 @@ def lib() -> ctypes.CDLL:
         _lib.ref_dsyrk.argtypes = [c_char, c_char, c_int64, c_int64, c_double, c_void_p, c_int64, c_double, c_void_p, c_int64]
         _lib.ref_ssyrk.argtypes = [c_char, c_char, c_int64, c_int64, c_float, c_void_p, c_int64, c_float, c_void_p, c_int64]
         _lib.ref_dsyrk.restype = _lib.ref_ssyrk.restype = c_int
+        tri = [c_char, c_char, c_char, c_char, c_int64, c_int64]
+        _lib.ref_dtrmm.argtypes = _lib.ref_dtrsm.argtypes = tri + [c_double, c_void_p, c_int64, c_void_p, c_int64]
+        _lib.ref_strmm.argtypes = _lib.ref_strsm.argtypes = tri + [c_float, c_void_p, c_int64, c_void_p, c_int64]
+        for fn in ("ref_dtrmm", "ref_dtrsm", "ref_strmm", "ref_strsm"):
+            getattr(_lib, fn).restype = c_int
         for fn in ("ref_dgemm", "ref_sgemm", "ref_dgemm_hi", "ref_sgemm_hi", "ref_zgemm", "ref_zgemm_hi",
                    "ref_num_threads"):
             getattr(_lib, fn).restype = c_int
@@ -282,3 +287,32 @@ def ref_gemm_strided_batched(transa, transb, m, n, k, alpha, A, lda, stride_a, B
     for b in range(batch):
         ref_gemm(transa, transb, m, n, k, alpha, A[b * stride_a:], lda, B[b * stride_b:], ldb, beta,
                  C[b * stride_c:], ldc)
+
+
+def _tri_call(which, side, uplo, trans, diag, m, n, alpha, A, lda, B, ldb) -> None:
+    dt = B.dtype
+    _flat(A, dt), _flat(B, dt)
+    if dt == np.float64:
+        fn, a = getattr(lib(), f"ref_d{which}"), float(alpha)
+    elif dt == np.float32:
+        fn, a = getattr(lib(), f"ref_s{which}"), float(np.float32(alpha))
+    else:
+        raise TypeError(f"unsupported dtype {dt}")
+    if m > 0 and n > 0:
+        _need(B, ldb, n, m, "B")
+        if alpha != 0:
+            na = m if side in "Ll" else n
+            _need(A, lda, na, na, "A")
+    rc = fn(_tr(side), _tr(uplo), _tr(trans), _tr(diag), m, n, a, A.ctypes.data, lda, B.ctypes.data, ldb)
+    if rc != 0:
+        raise ValueError(f"oracle rejected argument {-rc}")
+
+
+def ref_trmm(side, uplo, trans, diag, m, n, alpha, A, lda, B, ldb) -> None:
+    """B := alpha*op(A)*B (side L) or alpha*B*op(A) (side R), A triangular; B (flat storage) updated in place."""
+    _tri_call("trmm", side, uplo, trans, diag, m, n, alpha, A, lda, B, ldb)
+
+
+def ref_trsm(side, uplo, trans, diag, m, n, alpha, A, lda, B, ldb) -> None:
+    """Solve op(A)*X = alpha*B (side L) or X*op(A) = alpha*B (side R) by substitution; X overwrites B."""
+    _tri_call("trsm", side, uplo, trans, diag, m, n, alpha, A, lda, B, ldb)

@@ -354,3 +354,135 @@ int ref_sgemm_tf32(int terms, char transa, char transb, int64_t m, int64_t n, in
 
 DEFINE_REF_SYRK(ref_dsyrk, double)
 DEFINE_REF_SYRK(ref_ssyrk, float)
+
+/*
+ * Triangular level-3 routines (the paper names the level-3 BLAS as consumers of the GEMM kernel, Abstract and
+ * Introduction; their definitions are the BLAS ones).  A is a triangular matrix of order na (= m for side 'L',
+ * n for side 'R'); only the triangle named by uplo is read, and with diag = 'U' its diagonal is taken as 1
+ * without being read.  T = op(A) below is that triangular matrix, transposed for trans = 'T'.
+ *
+ *   TRMM:  B := alpha * T * B   (side L)      or   B := alpha * B * T   (side R)
+ *          every element is the sum over the non-zero part of the row/column of T, ascending index, one multiply
+ *          and one add per term, then one multiply by alpha.  Evaluated from a copy of B (the routine is in place).
+ *
+ *   TRSM:  solve T * X = alpha * B (side L)   or   X * T = alpha * B (side R);  X overwrites B.
+ *          Substitution, one unknown after the other in the order the triangle dictates:
+ *              x_i = (alpha * b_i - sum_{p already solved} T_ip x_p) / T_ii      (side L; side R alike on rows)
+ *          the sum taken in ascending p with one multiply and one add per term, subtracted once from alpha*b_i,
+ *          then one division (none for diag = 'U').  alpha == 0 gives X = 0 without reading A.
+ *
+ * t_elem returns T(i, p) for an effective position, 0 outside the triangle, 1 on a unit diagonal.
+ */
+#define DEFINE_REF_TRI(SUFFIX, T)                                                                          \
+  static T t_elem_##SUFFIX(const T* A, int64_t lda, int lower, int tr, int unit, int64_t i, int64_t p) {    \
+    /* (i, p) indexes T = op(A); the stored element is A(i, p) or, transposed, A(p, i) */                   \
+    const int64_t r = tr ? p : i, c = tr ? i : p;                                                           \
+    if (r == c) return unit ? (T)1 : A[r + c * lda];                                                        \
+    if (lower ? (r > c) : (r < c)) return A[r + c * lda];                                                   \
+    return (T)0;                                                                                            \
+  }                                                                                                         \
+  static int check_tri_##SUFFIX(char side, char uplo, char trans, char diag, int64_t m, int64_t n,          \
+                                int64_t lda, int64_t ldb) {                                                 \
+    const int left = (side == 'L' || side == 'l'), right = (side == 'R' || side == 'r');                    \
+    if (!left && !right) return 1;                                                                          \
+    if (!(uplo == 'L' || uplo == 'l' || uplo == 'U' || uplo == 'u')) return 2;                              \
+    if (!is_trans(trans) && !is_notrans(trans)) return 3;                                                   \
+    if (!(diag == 'U' || diag == 'u' || diag == 'N' || diag == 'n')) return 4;                              \
+    if (m < 0) return 5;                                                                                    \
+    if (n < 0) return 6;                                                                                    \
+    const int64_t na = left ? m : n;                                                                        \
+    if (lda < (na > 1 ? na : 1)) return 9;                                                                  \
+    if (ldb < (m > 1 ? m : 1)) return 11;                                                                   \
+    return 0;                                                                                               \
+  }                                                                                                         \
+  int ref_##SUFFIX##trmm(char side, char uplo, char trans, char diag, int64_t m, int64_t n, T alpha,        \
+                         const T* A, int64_t lda, T* B, int64_t ldb) {                                      \
+    const int bad = check_tri_##SUFFIX(side, uplo, trans, diag, m, n, lda, ldb);                            \
+    if (bad) return -bad;                                                                                   \
+    if (m == 0 || n == 0) return 0;                                                                         \
+    const int left = (side == 'L' || side == 'l'), lower = (uplo == 'L' || uplo == 'l');                    \
+    const int tr = is_trans(trans), unit = (diag == 'U' || diag == 'u');                                    \
+    if (alpha == (T)0) {                                                                                    \
+      for (int64_t j = 0; j < n; ++j)                                                                       \
+        for (int64_t i = 0; i < m; ++i) B[i + j * ldb] = (T)0;                                              \
+      return 0;                                                                                             \
+    }                                                                                                       \
+    T* old = (T*)malloc(sizeof(T) * (size_t)m * (size_t)n);                                                 \
+    if (!old) return -100;                                                                                  \
+    for (int64_t j = 0; j < n; ++j)                                                                         \
+      for (int64_t i = 0; i < m; ++i) old[i + j * m] = B[i + j * ldb];                                      \
+    const int eff_lower = (lower != tr); /* op(A) is lower triangular */                                    \
+    _Pragma("omp parallel for schedule(dynamic, 1)") for (int64_t j = 0; j < n; ++j) {                      \
+      for (int64_t i = 0; i < m; ++i) {                                                                     \
+        T acc = (T)0;                                                                                       \
+        if (left) { /* sum_p T(i,p) old(p,j): p <= i for lower T, p >= i for upper */                       \
+          const int64_t lo = eff_lower ? 0 : i, hi = eff_lower ? i + 1 : m;                                 \
+          for (int64_t p = lo; p < hi; ++p) {                                                               \
+            const T prod = t_elem_##SUFFIX(A, lda, lower, tr, unit, i, p) * old[p + j * m];                 \
+            acc = acc + prod;                                                                               \
+          }                                                                                                 \
+        } else { /* sum_p old(i,p) T(p,j): p >= j for lower T, p <= j for upper */                          \
+          const int64_t lo = eff_lower ? j : 0, hi = eff_lower ? n : j + 1;                                 \
+          for (int64_t p = lo; p < hi; ++p) {                                                               \
+            const T prod = old[i + p * m] * t_elem_##SUFFIX(A, lda, lower, tr, unit, p, j);                 \
+            acc = acc + prod;                                                                               \
+          }                                                                                                 \
+        }                                                                                                   \
+        B[i + j * ldb] = alpha * acc;                                                                       \
+      }                                                                                                     \
+    }                                                                                                       \
+    free(old);                                                                                              \
+    return 0;                                                                                               \
+  }                                                                                                         \
+  int ref_##SUFFIX##trsm(char side, char uplo, char trans, char diag, int64_t m, int64_t n, T alpha,        \
+                         const T* A, int64_t lda, T* B, int64_t ldb) {                                      \
+    const int bad = check_tri_##SUFFIX(side, uplo, trans, diag, m, n, lda, ldb);                            \
+    if (bad) return -bad;                                                                                   \
+    if (m == 0 || n == 0) return 0;                                                                         \
+    const int left = (side == 'L' || side == 'l'), lower = (uplo == 'L' || uplo == 'l');                    \
+    const int tr = is_trans(trans), unit = (diag == 'U' || diag == 'u');                                    \
+    if (alpha == (T)0) {                                                                                    \
+      for (int64_t j = 0; j < n; ++j)                                                                       \
+        for (int64_t i = 0; i < m; ++i) B[i + j * ldb] = (T)0;                                              \
+      return 0;                                                                                             \
+    }                                                                                                       \
+    const int eff_lower = (lower != tr);                                                                    \
+    if (left) { /* columns of B are independent systems T x = alpha b */                                    \
+      _Pragma("omp parallel for schedule(dynamic, 1)") for (int64_t j = 0; j < n; ++j) {                    \
+        T* x = &B[j * ldb];                                                                                 \
+        for (int64_t s = 0; s < m; ++s) {                                                                   \
+          const int64_t i = eff_lower ? s : m - 1 - s; /* forward for lower T, backward for upper */        \
+          const int64_t lo = eff_lower ? 0 : i + 1, hi = eff_lower ? i : m;                                 \
+          T acc = (T)0;                                                                                     \
+          for (int64_t p = lo; p < hi; ++p) {                                                               \
+            const T prod = t_elem_##SUFFIX(A, lda, lower, tr, unit, i, p) * x[p];                           \
+            acc = acc + prod;                                                                               \
+          }                                                                                                 \
+          const T rhs = alpha * x[i];                                                                       \
+          T v = rhs - acc;                                                                                  \
+          if (!unit) v = v / t_elem_##SUFFIX(A, lda, lower, tr, unit, i, i);                                \
+          x[i] = v;                                                                                         \
+        }                                                                                                   \
+      }                                                                                                     \
+    } else { /* rows of B are independent systems x^T T = alpha b^T: x_j needs x_p with T(p,j) != 0 */      \
+      _Pragma("omp parallel for schedule(dynamic, 16)") for (int64_t i = 0; i < m; ++i) {                   \
+        for (int64_t s = 0; s < n; ++s) {                                                                   \
+          const int64_t j = eff_lower ? n - 1 - s : s; /* upper T: forward over columns; lower: backward */ \
+          const int64_t lo = eff_lower ? j + 1 : 0, hi = eff_lower ? n : j;                                 \
+          T acc = (T)0;                                                                                     \
+          for (int64_t p = lo; p < hi; ++p) {                                                               \
+            const T prod = B[i + p * ldb] * t_elem_##SUFFIX(A, lda, lower, tr, unit, p, j);                 \
+            acc = acc + prod;                                                                               \
+          }                                                                                                 \
+          const T rhs = alpha * B[i + j * ldb];                                                             \
+          T v = rhs - acc;                                                                                  \
+          if (!unit) v = v / t_elem_##SUFFIX(A, lda, lower, tr, unit, j, j);                                \
+          B[i + j * ldb] = v;                                                                               \
+        }                                                                                                   \
+      }                                                                                                     \
+    }                                                                                                       \
+    return 0;                                                                                               \
+  }
+
+DEFINE_REF_TRI(d, double)
+DEFINE_REF_TRI(s, float)
