@@ -204,6 +204,32 @@ int b2_sgemm_strided_batched(char transa, char transb, int64_t m, int64_t n, int
                              float* C, int64_t ldc, int64_t stride_c, int64_t batch, void* cuda_stream);
 
 /*
+ * Triangular level-3 routines on the GEMM kernel (the paper names the level-3 BLAS as consumers of its kernel,
+ * Abstract and Introduction; the definitions are the BLAS ones).  A is triangular of order m (side 'L') or n
+ * (side 'R'); only the triangle named by uplo ('L'/'U') is read, and with diag = 'U' its diagonal is taken as 1
+ * and not read.  op(A) = A for transa 'N', A^T for 'T' (or 'C').
+ *     b2_dtrmm:  B := alpha*op(A)*B   (side 'L')   or   B := alpha*B*op(A)   (side 'R')
+ *     b2_dtrsm:  solve op(A)*X = alpha*B (side 'L') or X*op(A) = alpha*B (side 'R');  X overwrites B
+ * B is m x n, column-major, DEVICE memory, updated in place; A is DEVICE memory and is not modified.  alpha == 0
+ * sets B to zero without reading A.  No singularity test is made (a zero on the diagonal divides by zero).
+ * Method: recursive halving of the triangle puts all but the diagonal blocks of order <= 32 into calls of the
+ * GEMM kernel; a diagonal block is handled by a substitution / product kernel with one warp per right-hand side.
+ * The order of summation therefore differs from column-by-column substitution; results satisfy the componentwise
+ * residual bound of substitution, |op(A)*X - alpha*B| <= c*na*u*(|op(A)||X| + |alpha*B|), and are exact whenever
+ * all intermediate values are exactly representable.
+ * Argument numbering for -i: side 1, uplo 2, transa 3, diag 4, m 5, n 6, alpha 7, A 8, lda 9, B 10, ldb 11.
+ * Work is enqueued on cuda_stream; nothing is allocated.
+ */
+int b2_dtrmm(char side, char uplo, char transa, char diag, int64_t m, int64_t n, double alpha, const double* A,
+             int64_t lda, double* B, int64_t ldb, void* cuda_stream);
+int b2_strmm(char side, char uplo, char transa, char diag, int64_t m, int64_t n, float alpha, const float* A,
+             int64_t lda, float* B, int64_t ldb, void* cuda_stream);
+int b2_dtrsm(char side, char uplo, char transa, char diag, int64_t m, int64_t n, double alpha, const double* A,
+             int64_t lda, double* B, int64_t ldb, void* cuda_stream);
+int b2_strsm(char side, char uplo, char transa, char diag, int64_t m, int64_t n, float alpha, const float* A,
+             int64_t lda, float* B, int64_t ldb, void* cuda_stream);
+
+/*
  * Split-K GEMM for small m*n with long k.  One CTA per C tile leaves most SMs idle when m*n is small, however
  * long k is; here k is cut into `splits` contiguous chunks (whole 16-deep slabs), the chunks' partial products
  * are computed by one batched launch of the GEMM kernel into workspace planes, and a second kernel stores

@@ -36,6 +36,14 @@ _SIGNATURES = {
     "b2_zgemm4m": (c_int, [c_char, c_char, c_int64, c_int64, c_int64, ctypes.POINTER(c_double), c_void_p, c_int64,
                            c_void_p, c_int64, ctypes.POINTER(c_double), c_void_p, c_int64, c_void_p, c_size_t,
                            c_void_p]),
+    "b2_dtrmm": (c_int, [c_char, c_char, c_char, c_char, c_int64, c_int64, c_double, c_void_p, c_int64, c_void_p, c_int64,
+                         c_void_p]),
+    "b2_strmm": (c_int, [c_char, c_char, c_char, c_char, c_int64, c_int64, c_float, c_void_p, c_int64, c_void_p, c_int64,
+                         c_void_p]),
+    "b2_dtrsm": (c_int, [c_char, c_char, c_char, c_char, c_int64, c_int64, c_double, c_void_p, c_int64, c_void_p, c_int64,
+                         c_void_p]),
+    "b2_strsm": (c_int, [c_char, c_char, c_char, c_char, c_int64, c_int64, c_float, c_void_p, c_int64, c_void_p, c_int64,
+                         c_void_p]),
     "b2_gemm_splitk_auto": (c_int, [c_int64, c_int64, c_int64]),
     "b2_gemm_splitk_workspace_bytes": (c_size_t, [c_int, c_int64, c_int64, c_int64, c_int]),
     "b2_dgemm_splitk": (c_int, [c_char, c_char, c_int64, c_int64, c_int64, c_double, c_void_p, c_int64, c_void_p, c_int64,
@@ -189,6 +197,34 @@ def b2_zgemm4m(transa, transb, m, n, k, alpha, A, lda, B, ldb, beta, C, ldc, wor
     if check:
         _check("b2_zgemm4m", rc)
     return rc
+
+
+def _tri(which, side, uplo, trans, diag, m, n, alpha, A, lda, B, ldb, check) -> int:
+    dtype = next((t.dtype for t in (B, A) if t is not None), torch.float64)
+    if dtype == torch.float64:
+        name = f"b2_d{which}"
+    elif dtype == torch.float32:
+        name = f"b2_s{which}"
+    else:
+        raise TypeError(f"b2_{which} takes float64 or float32 tensors")
+    for t in (A, B):
+        if t is not None and (t.dtype != dtype or not t.is_cuda):
+            raise TypeError(f"b2_{which} takes CUDA tensors of one dtype")
+    rc = getattr(lib(), name)(_tr(side), _tr(uplo), _tr(trans), _tr(diag), m, n, alpha, _ptr(A), lda, _ptr(B), ldb,
+                              _stream())
+    if check:
+        _check(name, rc)
+    return rc
+
+
+def b2_trmm(side, uplo, trans, diag, m, n, alpha, A, lda, B, ldb, check=True) -> int:
+    """B := alpha*op(A)*B (side L) or alpha*B*op(A) (side R), A triangular; fp64 or fp32 by the tensors' dtype."""
+    return _tri("trmm", side, uplo, trans, diag, m, n, alpha, A, lda, B, ldb, check)
+
+
+def b2_trsm(side, uplo, trans, diag, m, n, alpha, A, lda, B, ldb, check=True) -> int:
+    """Solve op(A)*X = alpha*B (side L) or X*op(A) = alpha*B (side R), A triangular; X overwrites B."""
+    return _tri("trsm", side, uplo, trans, diag, m, n, alpha, A, lda, B, ldb, check)
 
 
 def b2_gemm_splitk_auto(m, n, k) -> int:
