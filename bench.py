@@ -147,6 +147,26 @@ def quick_gflops(fn, flops, iters=3, warm=3):
     return flops * iters / (e0.elapsed_time(e1) * 1e-3) / 1e9
 
 
+def graph_gflops(fn, flops, launches=20, replays=10):
+    """Throughput of `fn` replayed from a CUDA graph of `launches` back-to-back launches: the kernels' own time,
+    without the host's per-launch cost (which bounds problems that take only a few microseconds)."""
+    fn()
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        for _ in range(launches):
+            fn()
+    graph.replay()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(replays):
+        graph.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    return flops * launches * replays / (e0.elapsed_time(e1) * 1e-3) / 1e9
+
+
 def other_configs(b2, device):
     """Throughput of the remaining benchmark configurations (few launches each); reported inside the JSON line."""
     from paper_1611_08035_b200 import synth
@@ -161,6 +181,10 @@ def other_configs(b2, device):
         g = quick_gflops(lambda: fn(ta, tb, m, n, k, alpha, A, lda, B, ldb, beta, C, ldc), 2.0 * m * n * k)
         peak = FP64_PEAK_TFLOPS if kind == "d" else FP32_PEAK_TFLOPS
         row = {"workload": label, "gflops": round(g, 1), "frac_of_peak": round(g / 1e3 / peak, 4)}
+        if max(m, n, k) <= 1024 and not pad:  # microsecond-scale problems: also the kernel time without launch cost
+            gg = graph_gflops(lambda: fn(ta, tb, m, n, k, alpha, A, lda, B, ldb, beta, C, ldc), 2.0 * m * n * k)
+            row["gflops_graph_replay"] = round(gg, 1)
+            row["frac_of_peak_graph_replay"] = round(gg / 1e3 / peak, 4)
         if label.startswith("rank_k"):
             ms = 2.0 * m * n * k / g / 1e6
             row["hbm_gbs"] = round((2.0 * m * n + (m + n) * k) * 8 / (ms * 1e-3) / 1e9, 1)

@@ -1,4 +1,4 @@
-// fp64 DMMA kernels with TMA staging (variants 4-6): tensor-map encoding, launch, device status word.
+// fp64 DMMA kernels with TMA staging (variants 4-6, 8): tensor-map encoding, launch, device status word.
 #include <cuda.h>
 #include <cuda_runtime.h>
 
