@@ -41,6 +41,7 @@ def _pair(b2, oracle, ta, tb, m, n, k, alpha, beta, seed):
 def test_static_scratch_matches_workspace_entry_on_two_calls_in_a_row(b2, oracle):
     _pair(b2, oracle, "N", "N", 200, 150, 170, 1 + 0.5j, 0.25 - 0.75j, seed=901)
     _pair(b2, oracle, "T", "N", 130, 71, 33, 0.3 - 0.8j, 0j, seed=902)  # smaller planes over the stale contents
+    _pair(b2, oracle, "C", "T", 90, 40, 57, 1 - 1j, 0.5j, seed=903)     # a conjugate transpose
 
 
 def test_static_scratch_limit_and_argument_errors(b2):
@@ -49,7 +50,7 @@ def test_static_scratch_limit_and_argument_errors(b2):
     assert b2.b2_zgemm4m_workspace_bytes("N", "N", 512, 512, 512) > b2.ZGEMM4M_STATIC_BYTES
     assert b2.b2_zgemm4m_static("N", "N", 512, 512, 512, 1, z, 512, z, 512, 0, z, 512, check=False) == 1005
     assert "scratch" in b2.strerror(1005)
-    assert b2.b2_zgemm4m_static("C", "N", 4, 4, 4, 1, z, 4, z, 4, 0, z, 4, check=False) == -1
+    assert b2.b2_zgemm4m_static("X", "N", 4, 4, 4, 1, z, 4, z, 4, 0, z, 4, check=False) == -1
     assert b2.b2_zgemm4m_static("N", "N", 4, 4, 4, 1, z, 3, z, 4, 0, z, 4, check=False) == -8
     torch.cuda.synchronize()
     assert (z == 0).all()
