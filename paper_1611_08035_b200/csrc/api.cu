@@ -24,6 +24,7 @@ int launch_f32_v0(const GemmArgs<float>&, bool, bool, bool, cudaStream_t);
 int launch_f32_v1(const GemmArgs<float>&, bool, bool, bool, cudaStream_t);
 int launch_f32_v2(const GemmArgs<float>&, bool, bool, bool, cudaStream_t);
 int launch_f32_v3(const GemmArgs<float>&, bool, bool, bool, cudaStream_t);
+int launch_f32_s32(const GemmArgs<float>&, bool, bool, bool, cudaStream_t);
 
 namespace {
 
@@ -45,10 +46,11 @@ const LaunchFn<double> kF64Launch[] = {launch_f64_v0, launch_f64_v1, launch_f64_
 const VariantInfo kF32Info[] = {
     {"ffma2_128x128x16_s4", "ffma2", 128, 128, 16, 4, 256, 2, 0.72},
     {"ffma2_128x64x16_s4", "ffma2", 128, 64, 16, 4, 128, 3, 0.775},
-    {"ffma2_64x64x16_s4", "ffma2", 64, 64, 16, 4, 64, 6, 0.68},
+    {"ffma2_64x64x16_s4", "ffma2", 64, 64, 16, 4, 64, 6, 0.64},
     {"ffma_128x64x16_s4", "ffma", 128, 64, 16, 4, 128, 4, 0.70},
+    {"ffma2_t4_32x32x16_s4", "ffma2", 32, 32, 16, 4, 64, 8, 0.40},
 };
-const LaunchFn<float> kF32Launch[] = {launch_f32_v0, launch_f32_v1, launch_f32_v2, launch_f32_v3};
+const LaunchFn<float> kF32Launch[] = {launch_f32_v0, launch_f32_v1, launch_f32_v2, launch_f32_v3, launch_f32_s32};
 
 }  // namespace
 
@@ -119,17 +121,26 @@ static bool operands_aligned(const T* A, int64_t lda, const T* B, int64_t ldb) {
          (lda % VEC == 0) && (ldb % VEC == 0);
 }
 
-// `aligned`: A and B have 16-byte aligned columns, which the TMA-staged variants need.
+// `aligned`: A and B have 16-byte aligned columns (16-byte staging); the TMA-staged variants need that and a
+// single problem (`batch` <= 1).
 template <typename T>
 int choose_variant(int64_t m, int64_t n, int64_t k, bool aligned, int64_t batch = 1) {
+  const bool tma_ok = aligned && batch <= 1;
   const int count = variant_count_t<T>();
   TileChoice cand[16];
   for (int v = 0; v < count && v < 16; ++v) {
     const VariantInfo& vi = variant_info_t<T>(v);
     const bool comparison_only = strcmp(vi.micro, "dfma") == 0 || strcmp(vi.micro, "ffma") == 0;
     const bool needs_alignment = strcmp(vi.micro, "dmma_tma") == 0;
-    cand[v] = TileChoice{vi.bm, vi.bn, vi.bk, vi.threads, vi.ctas_per_sm, vi.efficiency,
-                         comparison_only || (needs_alignment && !aligned)};
+    double eff = vi.efficiency;
+    // Unaligned operands are staged in 8- or 4-byte pieces: twice to four times the staging instructions, which
+    // weigh the more the smaller the tile (staging work per multiply-add goes with (BM+BN)/(BM*BN)); measured on
+    // the 1001 x 999 x 1003 problem with odd leading dimensions.
+    if (!aligned) eff *= 1.0 - 3.2 * (double)(vi.bm + vi.bn) / ((double)vi.bm * vi.bn);
+    cand[v] = TileChoice{vi.bm, vi.bn, vi.bk, vi.threads, vi.ctas_per_sm, eff,
+                         comparison_only || (needs_alignment && !tma_ok)};
+    // measured: a TMA-staged CTA starts about 2 microseconds later than a cp.async one (512^3: 17.4 against 12.6 us)
+    if (needs_alignment) cand[v].extra_fixed_clks = 4500.0;
   }
   return select_tile(cand, count < 16 ? count : 16, m, n, k, sm_count_cached(), (int)sizeof(T), batch);
 }
@@ -144,7 +155,7 @@ int gemm_launch_checked(int variant, bool ta, bool tb, int64_t m, int64_t n, int
   constexpr int64_t kVec = 16 / (int64_t)sizeof(T);
   const bool aligned = operands_aligned(A, lda, B, ldb) &&
                        (ex.batch <= 1 || (ex.stride_a % kVec == 0 && ex.stride_b % kVec == 0));
-  if (variant == B2_VARIANT_AUTO) variant = choose_variant<T>(m, n, k, aligned && ex.batch <= 1, ex.batch);
+  if (variant == B2_VARIANT_AUTO) variant = choose_variant<T>(m, n, k, aligned, ex.batch);
   GemmArgs<T> args;
   args.m = m, args.n = n, args.k = k;
   args.alpha = alpha, args.beta = beta;

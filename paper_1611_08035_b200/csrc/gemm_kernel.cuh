@@ -339,7 +339,8 @@ struct DmmaMicro {
 // 16-byte shared-memory loads: 64 independent FMAs per outer product.
 // A warp is 8 lanes along m by 4 lanes along n, so it covers 64 x 32 of C.
 // ---------------------------------------------------------------------------------------
-template <typename T_, int BM_, int BN_, int BK_, int WARPS_M, int WARPS_N, bool TA, bool TB, bool PACKED = true>
+template <typename T_, int BM_, int BN_, int BK_, int WARPS_M, int WARPS_N, bool TA, bool TB, bool PACKED = true,
+          int TM_ = 8, int TN_ = 8>
 struct SimtMicro {
   using T = T_;
   // fp32 only: PACKED uses the pair instruction fma.rn.f32x2; false keeps scalar FFMA (comparison variant)
@@ -347,9 +348,11 @@ struct SimtMicro {
   static constexpr int BM = BM_, BN = BN_, BK = BK_;
   static constexpr int NT = 32 * WARPS_M * WARPS_N;
   static constexpr int VEC = 16 / sizeof(T);
-  static constexpr int TM = 8, TN = 8;
+  // per-thread block: 8 x 8 for large problems; 4 x 4 quadruples the warps per tile for small ones
+  static constexpr int TM = TM_, TN = TN_;
+  static_assert(TM % VEC == 0 && TN % VEC == 0 && TM % 2 == 0, "thread block must be whole 16-byte vectors");
   static constexpr int WTM = 8 * TM, WTN = 4 * TN;
-  static_assert(BM == WARPS_M * WTM && BN == WARPS_N * WTN, "CTA tile must be warps x (64 x 32)");
+  static_assert(BM == WARPS_M * WTM && BN == WARPS_N * WTN, "CTA tile must be warps x (8 TM x 4 TN)");
   static constexpr Layout LA = OC, LB = OC;
   static constexpr int PA = BM + VEC, PB = BN + VEC;
   static constexpr int A_STAGE = BK * PA, B_STAGE = BK * PB;

@@ -7,6 +7,7 @@
 // three "pipelines" a tile occupies -- the arithmetic pipe, the L2->shared-memory feed and the
 // C traffic of the epilogue -- and keep the candidate with the smallest estimate.
 #pragma once
+#include <math.h>
 #include <stdint.h>
 
 namespace b2 {
@@ -17,6 +18,7 @@ struct TileChoice {
   int ctas_per_sm;   // CTAs of this variant that fit on one SM
   double efficiency;  // measured steady-state fraction of the arithmetic pipe's peak
   bool explicit_only;  // never chosen automatically (comparison variants)
+  double extra_fixed_clks = 0.0;  // start-up cost beyond the common one (TMA: descriptor fetch, barrier set-up)
 };
 
 // Measured / derived machine rates per SM (B200): FP64 and FP32 multiply-adds per clock, the
@@ -47,23 +49,41 @@ inline double estimate_clks(const TileChoice& c, int64_t m, int64_t n, int64_t k
   // tiles are handed out CTA by CTA; an SM ends up with ceil(tiles / sms) of them
   const double per_sm = (double)(int64_t)((tiles + sms - 1) / sms);
   const double fma_tile = (double)c.bm * c.bn * c.bk * kt;
-  // arithmetic pipe
-  const double t_math = fma_tile / (r.fma_per_clk * c.efficiency);
-  // feed: bytes of A and B a tile pulls through L2 per multiply-add
-  const double feed_tile = (double)(c.bm + c.bn) * c.bk * kt * elem_bytes;
-  const double t_feed = feed_tile / r.l2_bytes_per_clk;
-  const double t_main = t_math > t_feed ? t_math : t_feed;
-  // epilogue: C read + write at the SM's share of HBM bandwidth
+  // The SM's tiles run ctas_per_sm at a time; the last, partial group runs with fewer resident warps.
+  const double cps = (double)c.ctas_per_sm;
+  const double full_groups = (double)(int64_t)(per_sm / cps);
+  const double rem = per_sm - full_groups * cps;  // tiles of the partial group (0 .. cps-1)
+  // `efficiency` is the measured fraction of the arithmetic pipe's peak with the SM fully populated by this
+  // variant; with fewer resident warps the pipe waits on latencies.  Measured with the 64 x 64 DMMA tile and
+  // cp.async staging: 4 warps on an SM reach about 0.6 of that, 8 warps 0.85, 16 warps all of it -- fitted by
+  // 1 - exp(-w/4.3).  TMA staging (no staging instructions, no CTA-wide barrier) loses less: 1 - exp(-w/3.3).
+  const double efold = c.extra_fixed_clks > 0.0 ? 3.3 : 4.3;
+  const double w_full = cps * c.threads / 32.0;
+  auto occupancy = [&](double ctas) {
+    return (1.0 - exp(-(ctas * c.threads / 32.0) / efold)) / (1.0 - exp(-w_full / efold));
+  };
+  // feed: bytes of A and B a tile pulls through L2; epilogue: C read + write at the SM's share of HBM bandwidth
+  const double t_feed = (double)(c.bm + c.bn) * c.bk * kt * elem_bytes / r.l2_bytes_per_clk;
   const double t_epi = 2.0 * c.bm * c.bn * elem_bytes / r.hbm_bytes_per_clk;
-  const double t_fixed = r.tile_fixed_clks + t_epi;
-  // With >= 2 resident CTAs one tile's ramp-up/epilogue overlaps another tile's main loop;
-  // with a single resident CTA every tile pays it.
-  const double resident = per_sm < c.ctas_per_sm ? per_sm : c.ctas_per_sm;
-  if (resident >= 2.0) {
-    const double overlapped = per_sm * (t_main > t_epi ? t_main : t_epi);
-    return overlapped + t_fixed;
+  const double t_fixed = r.tile_fixed_clks + c.extra_fixed_clks + t_epi;
+  auto tile_clks = [&](double occ) {
+    const double t_math = fma_tile / (r.fma_per_clk * c.efficiency * occ);
+    const double t_main = t_math > t_feed ? t_math : t_feed;
+    return t_main > t_epi ? t_main : t_epi;
+  };
+  if (per_sm < 2.0) return per_sm * (tile_clks(occupancy(1.0)) + t_fixed);  // nothing overlaps the fixed costs
+  double total = full_groups * cps * tile_clks(1.0);
+  if (rem > 0.0) {
+    double occ = occupancy(rem);
+    // A launch that fits in one wave starts all its CTAs together; doing identical work they stay in step and
+    // their waits coincide (measured: about 8 % slower than the same tiles dispatched one by one as others retire).
+    if (full_groups == 0.0 && rem >= 3.0) occ *= 0.92;
+    total += rem * tile_clks(occ);
+  } else if (full_groups == 1.0 && tiles <= (double)sms * cps) {
+    total /= 0.92;  // exactly one full wave: the same lock-step
   }
-  return per_sm * (t_main + t_fixed);
+  // with >= 2 tiles per SM one tile's ramp-up and epilogue overlap another tile's main loop: paid once
+  return total + t_fixed;
 }
 
 // Index of the candidate with the smallest estimate.
