@@ -6,8 +6,8 @@
 //     T = [T11  0 ; T21 T22] (lower):   X1 = solve(T11, B1);  B2 := alpha*B2 - T21*X1 (GEMM);  X2 = solve(T22, B2)
 //
 // and its mirror images for upper triangles, the right side and the products.  The recursion stops at diagonal
-// blocks of order <= 32, which a small kernel handles with one warp per right-hand side (or per row of B for
-// the right side): the block of T sits in shared memory, lane i of the warp owns unknown i.
+// blocks of order <= 128, which a small kernel handles with one warp per four right-hand sides (or rows of B
+// for the right side), 32 x 32 sub-block by sub-block.
 #include <cuda_runtime.h>
 
 #include "b2gemm.h"
@@ -16,39 +16,64 @@
 namespace b2 {
 namespace {
 
-constexpr int NB = 32;             // order of a leaf block = one warp: lane i owns unknown i
+constexpr int SUB = 32;            // a sub-block = one warp: lane i owns unknown i of the sub-block
+constexpr int NSUB = 4;            // sub-blocks per leaf
+constexpr int NB = SUB * NSUB;     // order of a leaf block (128)
 constexpr int LEAF_THREADS = 256;  // 8 warps
-constexpr int LEAF_VECS = 32;      // vectors per CTA (4 per warp)
+constexpr int VPW = 4;             // vectors per warp
+constexpr int LEAF_VECS = VPW * LEAF_THREADS / 32;  // vectors per CTA (32)
 
 bool t_is_n(char c) { return c == 'N' || c == 'n'; }
 bool t_is_t(char c) { return c == 'T' || c == 't' || c == 'C' || c == 'c'; }
 
-// One leaf: nvec independent vectors x of length nb (element i of vector v at X[i*si + v*sv]; one of si, sv is 1)
-// and the nb x nb triangular matrix M with M(i,p) = mt ? A(p,i) : A(i,p), lower triangular iff LOWER (the
-// caller passes the triangle as it looks after `mt`), unit diagonal iff unit.
+// One leaf: nvec independent vectors x of length nb <= 128 (element i of vector v at X[i*si + v*sv]; one of si,
+// sv is 1) and the nb x nb triangular matrix M with M(i,p) = mt ? A(p,i) : A(i,p), lower triangular iff LOWER
+// (the caller passes the triangle as it looks after `mt`), unit diagonal iff unit.
 //   SOLVE:  x := M^-1 * (alpha*x)          else:  x := alpha * M * x
-// A warp works on one vector at a time, lane i holding x_i; values travel between lanes by shuffle.  M is
-// padded to 32 x 32 with the identity and x with zeros.  The CTA's 32 vectors pass through a shared-memory
-// tile so that global loads and stores are coalesced whichever of si, sv is 1.
+// M is handled as 4 x 4 sub-blocks of order 32.  A warp holds four vectors, lane i owning element i of each
+// sub-block (16 values per lane); values travel between lanes by shuffle.  The CTA walks through the sub-blocks
+// of the triangle in dependency order -- solve (or multiply by) a diagonal sub-block, then apply the
+// off-diagonal sub-blocks of its block column (row) -- staging one 32 x 32 sub-block of M at a time in shared
+// memory.  M is padded with the identity and x with zeros beyond nb; sub-blocks wholly beyond nb are skipped.
+// The CTA's 32 vectors pass through a shared-memory tile so that global loads and stores are coalesced
+// whichever of si, sv is 1.
 template <typename T, bool SOLVE, bool LOWER>
-__global__ void __launch_bounds__(LEAF_THREADS)
+__global__ void __launch_bounds__(LEAF_THREADS, 2)
     tri_leaf_kernel(int nb, const T* __restrict__ A, int64_t lda, bool mt, bool unit, T alpha, T* __restrict__ X,
                     int64_t si, int64_t sv, int64_t nvec) {
-  __shared__ T Ms[NB * NB];               // Ms[p*NB + i] = M(i, p): a column of M is contiguous over lanes
+  __shared__ T Ms[SUB * SUB];             // Ms[p*SUB + i] = M(i, p) of the staged sub-block
   __shared__ T Xs[LEAF_VECS * (NB + 1)];  // Xs[v*(NB+1) + i]
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  for (int e = tid; e < NB * NB; e += LEAF_THREADS) {
-    const int i = e / NB, p = e % NB;  // logical M(i, p)
-    T v = (i == p) ? T(1) : T(0);
-    if (i < nb && p < nb) {
-      if (i == p) {
-        if (!unit) v = A[i + (int64_t)i * lda];
-      } else if (LOWER ? (i > p) : (i < p)) {
-        v = mt ? A[p + (int64_t)i * lda] : A[i + (int64_t)p * lda];
+  const int nsub = (nb + SUB - 1) / SUB;  // sub-blocks that hold anything
+
+  // Sub-block (bi, bj) of M travels global -> registers (fetch, issued one step ahead so that its latency hides
+  // behind the arithmetic of the current step) -> shared memory (commit, between two barriers).
+  constexpr int PER_THREAD = SUB * SUB / LEAF_THREADS;
+  T staged[PER_THREAD];
+  auto fetch = [&](int bi, int bj) {
+#pragma unroll
+    for (int u = 0; u < PER_THREAD; ++u) {
+      const int e = tid + u * LEAF_THREADS;
+      const int i = e % SUB, p = e / SUB;
+      const int gi = bi * SUB + i, gp = bj * SUB + p;
+      T v = (gi == gp) ? T(1) : T(0);
+      if (gi < nb && gp < nb) {
+        if (gi == gp) {
+          if (!unit) v = A[gi + (int64_t)gi * lda];
+        } else if (LOWER ? (gi > gp) : (gi < gp)) {
+          v = mt ? A[gp + (int64_t)gi * lda] : A[gi + (int64_t)gp * lda];
+        }
       }
+      staged[u] = v;
     }
-    Ms[p * NB + i] = v;
-  }
+  };
+  auto commit = [&]() {
+    __syncthreads();  // everybody is done with the previous sub-block
+#pragma unroll
+    for (int u = 0; u < PER_THREAD; ++u) Ms[tid + u * LEAF_THREADS] = staged[u];  // index p*SUB + i
+    __syncthreads();
+  };
+
   const int64_t v0 = blockIdx.x * (int64_t)LEAF_VECS;
   const bool elem_fastest = (si == 1);  // consecutive threads walk along whichever index is contiguous in memory
   for (int e = tid; e < LEAF_VECS * NB; e += LEAF_THREADS) {
@@ -59,29 +84,89 @@ __global__ void __launch_bounds__(LEAF_THREADS)
   }
   __syncthreads();
 
-  const T diag = Ms[lane * NB + lane];
-  for (int v = warp; v < LEAF_VECS; v += LEAF_THREADS / 32) {
-    T x = Xs[v * (NB + 1) + lane];
-    if (SOLVE) {
-      x = alpha * x;
-#pragma unroll 4
-      for (int s = 0; s < NB; ++s) {
-        const int i = LOWER ? s : NB - 1 - s;  // forward for a lower M, backward for an upper one
-        if (lane == i) x = x / diag;
-        const T xi = __shfl_sync(0xffffffffu, x, i);
-        if (LOWER ? (lane > i) : (lane < i)) x -= Ms[i * NB + lane] * xi;  // M(lane, i)
-      }
-    } else {
-      T acc = T(0);
-#pragma unroll 4
-      for (int p = 0; p < NB; ++p) {
-        const T xp = __shfl_sync(0xffffffffu, x, p);
-        if (LOWER ? (p <= lane) : (p >= lane)) acc += Ms[p * NB + lane] * xp;  // M(lane, p)
-      }
-      x = alpha * acc;
-    }
-    Xs[v * (NB + 1) + lane] = x;
+  T x[VPW][NSUB];
+#pragma unroll
+  for (int q = 0; q < VPW; ++q)
+#pragma unroll
+    for (int b = 0; b < NSUB; ++b) x[q][b] = Xs[(warp * VPW + q) * (NB + 1) + b * SUB + lane];
+  if (SOLVE) {
+#pragma unroll
+    for (int q = 0; q < VPW; ++q)
+#pragma unroll
+      for (int b = 0; b < NSUB; ++b) x[q][b] = alpha * x[q][b];
   }
+
+  // Steps (sb, tb), tb >= sb.  SOLVE: sub-block blk(sb) is solved at tb == sb, then leaves sub-block blk(tb).
+  // Product: row blk(sb) is formed from its diagonal sub-block (tb == sb) and the sub-blocks blk(tb) whose old
+  // values it still needs; a lower M goes bottom-up so that those are still unchanged.
+  auto blk = [](int s) { return (SOLVE == LOWER) ? s : NSUB - 1 - s; };
+  auto fetch_step = [&](int sb, int tb) {
+    if (SOLVE) fetch(blk(tb), blk(sb)); else fetch(blk(sb), blk(tb));
+  };
+  T acc[VPW];
+  fetch_step(0, 0);
+#pragma unroll
+  for (int sb = 0; sb < NSUB; ++sb) {
+#pragma unroll
+    for (int tb = sb; tb < NSUB; ++tb) {
+      commit();
+      if (tb + 1 < NSUB) fetch_step(sb, tb + 1);
+      else if (sb + 1 < NSUB) fetch_step(sb + 1, sb + 1);
+      const int bs = blk(sb), bt = blk(tb);
+      if (bs >= nsub || bt >= nsub) continue;  // nothing but padding (uniform over the CTA)
+      if (SOLVE) {
+        if (tb == sb) {
+          const T diag = Ms[lane * SUB + lane];
+#pragma unroll 2
+          for (int s = 0; s < SUB; ++s) {
+            const int i = LOWER ? s : SUB - 1 - s;  // forward within a lower sub-block, backward within an upper
+            const T mi = Ms[i * SUB + lane];        // M(lane, i)
+#pragma unroll
+            for (int q = 0; q < VPW; ++q) {         // four independent chains
+              if (lane == i) x[q][bs] = x[q][bs] / diag;
+              const T xi = __shfl_sync(0xffffffffu, x[q][bs], i);
+              if (LOWER ? (lane > i) : (lane < i)) x[q][bs] -= mi * xi;
+            }
+          }
+        } else {
+#pragma unroll
+          for (int q = 0; q < VPW; ++q) acc[q] = T(0);
+#pragma unroll 4
+          for (int p = 0; p < SUB; ++p) {
+            const T mp = Ms[p * SUB + lane];  // M(lane of sub-block bt, p of sub-block bs)
+#pragma unroll
+            for (int q = 0; q < VPW; ++q) acc[q] += mp * __shfl_sync(0xffffffffu, x[q][bs], p);
+          }
+#pragma unroll
+          for (int q = 0; q < VPW; ++q) x[q][bt] -= acc[q];
+        }
+      } else {
+        if (tb == sb) {
+#pragma unroll
+          for (int q = 0; q < VPW; ++q) acc[q] = T(0);
+        }
+#pragma unroll 4
+        for (int p = 0; p < SUB; ++p) {
+          const T mp = Ms[p * SUB + lane];
+          const bool inside = (tb != sb) || (LOWER ? (p <= lane) : (p >= lane));
+#pragma unroll
+          for (int q = 0; q < VPW; ++q) {
+            const T xp = __shfl_sync(0xffffffffu, x[q][bt], p);
+            if (inside) acc[q] += mp * xp;
+          }
+        }
+      }
+    }
+    if (!SOLVE && blk(sb) < nsub) {
+#pragma unroll
+      for (int q = 0; q < VPW; ++q) x[q][blk(sb)] = alpha * acc[q];
+    }
+  }
+
+#pragma unroll
+  for (int q = 0; q < VPW; ++q)
+#pragma unroll
+    for (int b = 0; b < NSUB; ++b) Xs[(warp * VPW + q) * (NB + 1) + b * SUB + lane] = x[q][b];
   __syncthreads();
   for (int e = tid; e < LEAF_VECS * NB; e += LEAF_THREADS) {
     const int v = elem_fastest ? e / NB : e % LEAF_VECS, i = elem_fastest ? e % NB : e / LEAF_VECS;
