@@ -75,12 +75,12 @@ inline double estimate_clks(const TileChoice& c, int64_t m, int64_t n, int64_t k
   double total = full_groups * cps * tile_clks(1.0);
   if (rem > 0.0) {
     double occ = occupancy(rem);
-    // A launch that fits in one wave starts all its CTAs together; doing identical work they stay in step and
-    // their waits coincide (measured: about 8 % slower than the same tiles dispatched one by one as others retire).
+    // Measured: the tiles of a launch that fits in one wave take about 8 % longer than the same tiles in a long
+    // launch, where CTAs are dispatched one by one as others retire.
     if (full_groups == 0.0 && rem >= 3.0) occ *= 0.92;
     total += rem * tile_clks(occ);
   } else if (full_groups == 1.0 && tiles <= (double)sms * cps) {
-    total /= 0.92;  // exactly one full wave: the same lock-step
+    total /= 0.92;  // exactly one full wave: the same
   }
   // with >= 2 tiles per SM one tile's ramp-up and epilogue overlap another tile's main loop: paid once
   return total + t_fixed;
