@@ -50,36 +50,62 @@ __device__ __forceinline__ float tf32_rna(float x) {
 // P[i][p] for i < rows, p < kpad (pitch = terms*kpad floats): element (i, p) of op(X) rounded to TF32, zero for
 // p >= k.  x_is_k_contiguous: op(X)(i, p) = X[p + i*ld], else X[i + p*ld].  For terms == 3 the three column blocks
 // hold (hi, hi, lo) when lo_last, (hi, lo, hi) otherwise.
+// 64 x 64 tile per CTA of 256 threads, 16-byte loads along whichever index is contiguous in the source (when base
+// and leading dimension allow) and 16-byte stores along p: the pass is HBM-bound, so what matters is bytes in flight.
 template <bool K_CONTIG>
-__global__ void tf32_pack_kernel(const float* __restrict__ X, int64_t ld, int64_t rows, int64_t k, int64_t kpad,
-                                 int terms, bool lo_last, float* __restrict__ P) {
-  __shared__ float tile[32][33];
-  const int64_t i0 = (int64_t)blockIdx.y * 32, p0 = (int64_t)blockIdx.x * 32;
-  const int tx = threadIdx.x, ty = threadIdx.y;  // 32 x 8
+__global__ void __launch_bounds__(256)
+    tf32_pack_kernel(const float* __restrict__ X, int64_t ld, int64_t rows, int64_t k, int64_t kpad, int terms,
+                     bool lo_last, float* __restrict__ P) {
+  constexpr int TP = 64;
+  __shared__ float tile[TP][TP + 1];  // tile[i][p]
+  const int64_t i0 = (int64_t)blockIdx.y * TP, p0 = (int64_t)blockIdx.x * TP;
+  const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;  // 16 x 16
   const int64_t pitch = (int64_t)terms * kpad;
-  if (K_CONTIG) {
-    for (int r = ty; r < 32; r += 8) {
-      const int64_t i = i0 + r, p = p0 + tx;
-      tile[r][tx] = (i < rows && p < k) ? X[p + i * ld] : 0.0f;
+  const bool vec_ok = ((reinterpret_cast<uintptr_t>(X) & 15) == 0) && (ld % 4 == 0);
+  // c = index along the source's contiguous direction (p when K_CONTIG, else i), s = the other one
+  const int64_t c_base = K_CONTIG ? p0 : i0, s_base = K_CONTIG ? i0 : p0;
+  const int64_t c_end = K_CONTIG ? k : rows, s_end = K_CONTIG ? rows : k;
+#pragma unroll
+  for (int it = 0; it < TP / 16; ++it) {
+    const int sl = ty + it * 16, cl = tx * 4;
+    const int64_t sg = s_base + sl, cg = c_base + cl;
+    float v[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+    if (sg < s_end) {
+      const float* src = X + cg + sg * ld;
+      if (vec_ok && cg + 3 < c_end) {
+        const float4 q = *reinterpret_cast<const float4*>(src);
+        v[0] = q.x, v[1] = q.y, v[2] = q.z, v[3] = q.w;
+      } else {
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+          if (cg + e < c_end) v[e] = src[e];
+      }
     }
-  } else {
-    for (int r = ty; r < 32; r += 8) {  // r runs along p, tx along i (contiguous in the source)
-      const int64_t i = i0 + tx, p = p0 + r;
-      tile[tx][r] = (i < rows && p < k) ? X[i + p * ld] : 0.0f;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      if (K_CONTIG) tile[sl][cl + e] = v[e]; else tile[cl + e][sl] = v[e];
     }
   }
   __syncthreads();
-  for (int r = ty; r < 32; r += 8) {
-    const int64_t i = i0 + r, p = p0 + tx;
-    if (i >= rows || p >= kpad) continue;
-    const float x = tile[r][tx];
-    const float hi = tf32_rna(x);
-    float* row = P + i * pitch;
-    row[p] = hi;
+#pragma unroll
+  for (int it = 0; it < TP / 16; ++it) {
+    const int r = ty + it * 16;
+    const int64_t i = i0 + r, p = p0 + tx * 4;
+    if (i >= rows || p >= kpad) continue;  // kpad is a multiple of 32: a group of four is inside or outside as a whole
+    float hi[4], lo[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const float x = tile[r][tx * 4 + e];
+      hi[e] = tf32_rna(x);
+      lo[e] = tf32_rna(x - hi[e]);
+    }
+    float* row = P + i * pitch + p;
+    const float4 vh = make_float4(hi[0], hi[1], hi[2], hi[3]);
+    *reinterpret_cast<float4*>(row) = vh;
     if (terms == 3) {
-      const float lo = tf32_rna(x - hi);
-      row[kpad + p] = lo_last ? hi : lo;
-      row[2 * kpad + p] = lo_last ? lo : hi;
+      const float4 vl = make_float4(lo[0], lo[1], lo[2], lo[3]);
+      *reinterpret_cast<float4*>(row + kpad) = lo_last ? vh : vl;
+      *reinterpret_cast<float4*>(row + 2 * kpad) = lo_last ? vl : vh;
     }
   }
 }
@@ -369,8 +395,8 @@ int sgemm_tf32(int terms, char transa, char transb, int64_t m, int64_t n, int64_
   }
 
   // step 1: pack.  op(A)(i, p): A[i + p*lda] (N) or A[p + i*lda] (T);  op(B)^T(j, p): B[p + j*ldb] (N) or B[j + p*ldb] (T)
-  const dim3 pb(32, 8);
-  const dim3 ga((unsigned)(pl.kpad / 32), (unsigned)((m + 31) / 32)), gb((unsigned)(pl.kpad / 32), (unsigned)((n + 31) / 32));
+  const dim3 pb(256);
+  const dim3 ga((unsigned)((pl.kpad + 63) / 64), (unsigned)((m + 63) / 64)), gb((unsigned)((pl.kpad + 63) / 64), (unsigned)((n + 63) / 64));
   if (t_is_n(transa))
     tf32_pack_kernel<false><<<ga, pb, 0, st>>>(A, lda, m, k, pl.kpad, terms, true, PA);
   else
