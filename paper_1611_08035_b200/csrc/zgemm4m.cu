@@ -12,6 +12,9 @@
 namespace b2 {
 namespace {
 
+// The element-wise kernels below run on a 2-D grid: blockIdx.x walks down a column in steps of the block size,
+// blockIdx.y (with a stride loop, the grid's second extent is limited) over columns; no integer division per element.
+
 // planes[0] = alpha_r*re - alpha_i*im, planes[1] = alpha_r*im + alpha_i*re of a rows x cols
 // interleaved complex matrix with leading dimension ld (complex elements); plane pitch ldp.
 // conj: the element is conjugated first (a conjugate transpose = plain transpose of these planes).
@@ -19,21 +22,29 @@ namespace {
 __global__ void zsplit_scale_kernel(int64_t rows, int64_t cols, const double2* __restrict__ X, int64_t ld, double sr,
                                     double si, bool conj, double* __restrict__ Pr, double* __restrict__ Pi,
                                     double* __restrict__ Ps, int64_t ldp) {
-  const int64_t total = rows * cols;
-  for (int64_t idx = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; idx < total;
-       idx += (int64_t)gridDim.x * blockDim.x) {
-    const int64_t r = idx % rows, c = idx / rows;
-    double2 v = X[r + c * ld];
-    if (conj) v.y = -v.y;
-    double pr = v.x, pi = v.y;
-    if (!(sr == 1.0 && si == 0.0)) {
-      pr = sr * v.x - si * v.y;
-      pi = sr * v.y + si * v.x;
+  const bool plain = (sr == 1.0 && si == 0.0);
+  for (int64_t c = blockIdx.y; c < cols; c += gridDim.y) {
+    const double2* x = X + c * ld;
+    for (int64_t r = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; r < rows; r += (int64_t)gridDim.x * blockDim.x) {
+      double2 v = x[r];
+      if (conj) v.y = -v.y;
+      double pr = v.x, pi = v.y;
+      if (!plain) {
+        pr = sr * v.x - si * v.y;
+        pi = sr * v.y + si * v.x;
+      }
+      Pr[r + c * ldp] = pr;
+      Pi[r + c * ldp] = pi;
+      if (Ps) Ps[r + c * ldp] = pr + pi;
     }
-    Pr[r + c * ldp] = pr;
-    Pi[r + c * ldp] = pi;
-    if (Ps) Ps[r + c * ldp] = pr + pi;
   }
+}
+
+__global__ void zmerge_kernel(int64_t rows, int64_t cols, const double* __restrict__ Pr,
+                              const double* __restrict__ Pi, int64_t ldp, double2* __restrict__ X, int64_t ld) {
+  for (int64_t c = blockIdx.y; c < cols; c += gridDim.y)
+    for (int64_t r = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; r < rows; r += (int64_t)gridDim.x * blockDim.x)
+      X[r + c * ld] = make_double2(Pr[r + c * ldp], Pi[r + c * ldp]);
 }
 
 // 3M: C := ((beta*C)r + T1 - T2,  ((beta*C)i - T1 - T2) + T3), the additions in exactly this order;
@@ -41,54 +52,44 @@ __global__ void zsplit_scale_kernel(int64_t rows, int64_t cols, const double2* _
 __global__ void zmerge3m_kernel(int64_t rows, int64_t cols, const double* __restrict__ T1,
                                 const double* __restrict__ T2, const double* __restrict__ T3, int64_t ldp, double br,
                                 double bi, double2* __restrict__ X, int64_t ld) {
-  const int64_t total = rows * cols;
   const bool zero = (br == 0.0 && bi == 0.0);
-  for (int64_t idx = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; idx < total;
-       idx += (int64_t)gridDim.x * blockDim.x) {
-    const int64_t r = idx % rows, c = idx / rows;
-    double cr = 0.0, ci = 0.0;
-    if (!zero) {
-      const double2 v = X[r + c * ld];
-      cr = br * v.x - bi * v.y;
-      ci = br * v.y + bi * v.x;
+  for (int64_t c = blockIdx.y; c < cols; c += gridDim.y) {
+    for (int64_t r = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; r < rows; r += (int64_t)gridDim.x * blockDim.x) {
+      double cr = 0.0, ci = 0.0;
+      if (!zero) {
+        const double2 v = X[r + c * ld];
+        cr = br * v.x - bi * v.y;
+        ci = br * v.y + bi * v.x;
+      }
+      const double t1 = T1[r + c * ldp], t2 = T2[r + c * ldp], t3 = T3[r + c * ldp];
+      X[r + c * ld] = make_double2((cr + t1) - t2, ((ci - t1) - t2) + t3);
     }
-    const double t1 = T1[r + c * ldp], t2 = T2[r + c * ldp], t3 = T3[r + c * ldp];
-    X[r + c * ld] = make_double2((cr + t1) - t2, ((ci - t1) - t2) + t3);
-  }
-}
-
-__global__ void zmerge_kernel(int64_t rows, int64_t cols, const double* __restrict__ Pr,
-                              const double* __restrict__ Pi, int64_t ldp, double2* __restrict__ X, int64_t ld) {
-  const int64_t total = rows * cols;
-  for (int64_t idx = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; idx < total;
-       idx += (int64_t)gridDim.x * blockDim.x) {
-    const int64_t r = idx % rows, c = idx / rows;
-    X[r + c * ld] = make_double2(Pr[r + c * ldp], Pi[r + c * ldp]);
   }
 }
 
 // C := beta*C (complex); beta == 0 stores zeros without reading C.
 __global__ void zscale_kernel(int64_t rows, int64_t cols, double br, double bi, double2* __restrict__ X, int64_t ld) {
-  const int64_t total = rows * cols;
   const bool zero = (br == 0.0 && bi == 0.0);
-  for (int64_t idx = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; idx < total;
-       idx += (int64_t)gridDim.x * blockDim.x) {
-    const int64_t r = idx % rows, c = idx / rows;
-    double2* x = X + r + c * ld;
-    if (zero) {
-      *x = make_double2(0.0, 0.0);
-    } else {
-      const double2 v = *x;
-      *x = make_double2(br * v.x - bi * v.y, br * v.y + bi * v.x);
+  for (int64_t c = blockIdx.y; c < cols; c += gridDim.y) {
+    for (int64_t r = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; r < rows; r += (int64_t)gridDim.x * blockDim.x) {
+      double2* x = X + r + c * ld;
+      if (zero) {
+        *x = make_double2(0.0, 0.0);
+      } else {
+        const double2 v = *x;
+        *x = make_double2(br * v.x - bi * v.y, br * v.y + bi * v.x);
+      }
     }
   }
 }
 
-unsigned grid_for(int64_t total) {
-  int64_t blocks = (total + 255) / 256;
-  if (blocks > 148 * 16) blocks = 148 * 16;
-  if (blocks < 1) blocks = 1;
-  return (unsigned)blocks;
+// grid for a rows x cols element-wise pass with 256-thread blocks
+dim3 grid_for(int64_t rows, int64_t cols) {
+  int64_t gx = (rows + 255) / 256;
+  if (gx > 64) gx = 64;
+  if (gx < 1) gx = 1;
+  int64_t gy = cols < 1 ? 1 : (cols > 16384 ? 16384 : cols);
+  return dim3((unsigned)gx, (unsigned)gy, 1);
 }
 
 struct Plan {
@@ -147,7 +148,7 @@ extern "C" int b2_zgemm4m(char transa, char transb, int64_t m, int64_t n, int64_
   double2* Cz = static_cast<double2*>(C);
   if (scale_only) {
     if (br == 1.0 && bi == 0.0) return B2_OK;
-    zscale_kernel<<<grid_for(m * n), 256, 0, st>>>(m, n, br, bi, Cz, ldc);
+    zscale_kernel<<<grid_for(m, n), 256, 0, st>>>(m, n, br, bi, Cz, ldc);
     return cudaGetLastError() == cudaSuccess ? B2_OK : B2_ERR_LAUNCH;
   }
   const Plan p = make_plan(transa, transb, m, n, k);
@@ -161,13 +162,13 @@ extern "C" int b2_zgemm4m(char transa, char transb, int64_t m, int64_t n, int64_
   double* Cr = reinterpret_cast<double*>(w + p.off[4]);
   double* Ci = reinterpret_cast<double*>(w + p.off[5]);
 
-  zsplit_scale_kernel<<<grid_for(p.ra * p.ca), 256, 0, st>>>(p.ra, p.ca, static_cast<const double2*>(A), lda, ar, ai,
+  zsplit_scale_kernel<<<grid_for(p.ra, p.ca), 256, 0, st>>>(p.ra, p.ca, static_cast<const double2*>(A), lda, ar, ai,
                                                            is_c(transa), Apr, Api, nullptr, p.lpa);
-  zsplit_scale_kernel<<<grid_for(p.rb * p.cb), 256, 0, st>>>(p.rb, p.cb, static_cast<const double2*>(B), ldb, 1.0,
+  zsplit_scale_kernel<<<grid_for(p.rb, p.cb), 256, 0, st>>>(p.rb, p.cb, static_cast<const double2*>(B), ldb, 1.0,
                                                            0.0, is_c(transb), Br, Bi, nullptr, p.lpb);
   double first_beta = 0.0;
   if (!beta0) {
-    zsplit_scale_kernel<<<grid_for(m * n), 256, 0, st>>>(m, n, Cz, ldc, br, bi, false, Cr, Ci, nullptr, p.lpc);
+    zsplit_scale_kernel<<<grid_for(m, n), 256, 0, st>>>(m, n, Cz, ldc, br, bi, false, Cr, Ci, nullptr, p.lpc);
     first_beta = 1.0;
   }
   transa = real_op(transa), transb = real_op(transb);
@@ -183,7 +184,7 @@ extern "C" int b2_zgemm4m(char transa, char transb, int64_t m, int64_t n, int64_
   if (rc) return rc;
   rc = gemm_entry<double>(B2_VARIANT_AUTO, transa, transb, m, n, k, 1.0, Api, p.lpa, Br, p.lpb, 1.0, Ci, p.lpc, st);
   if (rc) return rc;
-  zmerge_kernel<<<grid_for(m * n), 256, 0, st>>>(m, n, Cr, Ci, p.lpc, Cz, ldc);
+  zmerge_kernel<<<grid_for(m, n), 256, 0, st>>>(m, n, Cr, Ci, p.lpc, Cz, ldc);
   return cudaGetLastError() == cudaSuccess ? B2_OK : B2_ERR_LAUNCH;
 }
 
@@ -214,7 +215,7 @@ extern "C" int b2_zgemm3m(char transa, char transb, int64_t m, int64_t n, int64_
   double2* Cz = static_cast<double2*>(C);
   if (scale_only) {
     if (br == 1.0 && bi == 0.0) return B2_OK;
-    zscale_kernel<<<grid_for(m * n), 256, 0, st>>>(m, n, br, bi, Cz, ldc);
+    zscale_kernel<<<grid_for(m, n), 256, 0, st>>>(m, n, br, bi, Cz, ldc);
     return cudaGetLastError() == cudaSuccess ? B2_OK : B2_ERR_LAUNCH;
   }
   const Plan p = make_plan(transa, transb, m, n, k);
@@ -230,9 +231,9 @@ extern "C" int b2_zgemm3m(char transa, char transb, int64_t m, int64_t n, int64_
     Bp[i] = reinterpret_cast<double*>(w + 3 * p.sa + i * p.sb);
     T[i] = reinterpret_cast<double*>(w + 3 * p.sa + 3 * p.sb + i * p.sc);
   }
-  zsplit_scale_kernel<<<grid_for(p.ra * p.ca), 256, 0, st>>>(p.ra, p.ca, static_cast<const double2*>(A), lda, ar, ai,
+  zsplit_scale_kernel<<<grid_for(p.ra, p.ca), 256, 0, st>>>(p.ra, p.ca, static_cast<const double2*>(A), lda, ar, ai,
                                                            is_c(transa), Ap[0], Ap[1], Ap[2], p.lpa);
-  zsplit_scale_kernel<<<grid_for(p.rb * p.cb), 256, 0, st>>>(p.rb, p.cb, static_cast<const double2*>(B), ldb, 1.0,
+  zsplit_scale_kernel<<<grid_for(p.rb, p.cb), 256, 0, st>>>(p.rb, p.cb, static_cast<const double2*>(B), ldb, 1.0,
                                                            0.0, is_c(transb), Bp[0], Bp[1], Bp[2], p.lpb);
   if (cudaGetLastError() != cudaSuccess) return B2_ERR_LAUNCH;
   const char ta = real_op(transa), tb = real_op(transb);
@@ -241,7 +242,7 @@ extern "C" int b2_zgemm3m(char transa, char transb, int64_t m, int64_t n, int64_
                                       p.lpc, st);
     if (rc) return rc;
   }
-  zmerge3m_kernel<<<grid_for(m * n), 256, 0, st>>>(m, n, T[0], T[1], T[2], p.lpc, br, bi, Cz, ldc);
+  zmerge3m_kernel<<<grid_for(m, n), 256, 0, st>>>(m, n, T[0], T[1], T[2], p.lpc, br, bi, Cz, ldc);
   return cudaGetLastError() == cudaSuccess ? B2_OK : B2_ERR_LAUNCH;
 }
 
