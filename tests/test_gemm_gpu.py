@@ -345,3 +345,28 @@ def test_pipe_probe_rates(b2):
     f = pipes.probe("ffma", 256, 1, 4000)
     assert 55 <= d["fma_per_clk_per_sm"] <= 66 and 55 <= t["fma_per_clk_per_sm"] <= 66
     assert 110 <= f["fma_per_clk_per_sm"] <= 132
+
+
+@pytest.mark.parametrize("kind", ["d", "s"])
+def test_more_than_2_31_elements_of_c(b2, oracle, kind):
+    """C with more than 2^31 elements (46400^2): column offsets no longer fit 32 bits even in elements.  k is short,
+    so the run is cheap; the oracle evaluates a column sample (first, last, tile edges, around the 2^31-th element)
+    on the compacted problem, which is the same arithmetic column by column."""
+    tdt = torch.float64 if kind == "d" else torch.float32
+    m = n = 46400
+    k = 24
+    assert m * n > 2 ** 31
+    A, lda, B, ldb, _, _ = synth.gemm_inputs("N", "N", m, n, k, "int9", 9100, tdt)
+    C = torch.full((m * n,), 7.0, dtype=tdt, device="cuda")
+    fn = b2.b2_dgemm if kind == "d" else b2.b2_sgemm
+    fn("N", "N", m, n, k, 1.5, A.cuda(), lda, B.cuda(), ldb, 0.5, C, m)
+    assert b2.b2_device_status() == 0
+    edge = (2 ** 31) // m  # the column that holds element number 2^31
+    cols = sorted({0, 1, 63, 64, edge - 1, edge, edge + 1, n - 65, n - 64, n - 2, n - 1})
+    Bn = B.numpy().reshape(n, ldb)[cols].copy().reshape(-1)
+    want = np.full(m * len(cols), 7.0, dtype=A.numpy().dtype)
+    oracle.ref_gemm("N", "N", m, len(cols), k, 1.5, A.numpy(), lda, Bn, ldb, 0.5, want, m)
+    got = torch.stack([C[c * m:(c + 1) * m] for c in cols]).cpu().numpy().reshape(-1)
+    assert got.tobytes() == want.tobytes()
+    # nothing else moved: every element is an integer multiple of 0.5 within the range the data allow
+    assert float(C.abs().max()) <= 1.5 * 16 * k + 3.5
