@@ -44,11 +44,11 @@ const LaunchFn<double> kF64Launch[] = {launch_f64_v0, launch_f64_v1, launch_f64_
                                        launch_f64_v4, launch_f64_v5, launch_f64_v6, launch_f64_t32,
                                        launch_f64_tma_t32};
 const VariantInfo kF32Info[] = {
-    {"ffma2_128x128x16_s4", "ffma2", 128, 128, 16, 4, 256, 2, 0.72},
+    {"ffma2_t16x8_128x128x16_s3", "ffma2", 128, 128, 16, 3, 128, 2, 0.78, 16, 8, 3500.0},
     {"ffma2_128x64x16_s4", "ffma2", 128, 64, 16, 4, 128, 3, 0.775},
     {"ffma2_64x64x16_s4", "ffma2", 64, 64, 16, 4, 64, 6, 0.64},
     {"ffma_128x64x16_s4", "ffma", 128, 64, 16, 4, 128, 4, 0.70},
-    {"ffma2_t4_32x32x16_s4", "ffma2", 32, 32, 16, 4, 64, 8, 0.40},
+    {"ffma2_t4_32x32x16_s4", "ffma2", 32, 32, 16, 4, 64, 8, 0.40, 4, 4},
 };
 const LaunchFn<float> kF32Launch[] = {launch_f32_v0, launch_f32_v1, launch_f32_v2, launch_f32_v3, launch_f32_s32};
 
@@ -123,8 +123,11 @@ static bool operands_aligned(const T* A, int64_t lda, const T* B, int64_t ldb) {
 
 // `aligned`: A and B have 16-byte aligned columns (16-byte staging); the TMA-staged variants need that and a
 // single problem (`batch` <= 1).
+// ta / tb: op(A) = A^T, op(B) = B^T.  They matter to the FMA micro-kernels only, which want both operands packed
+// with the C index contiguous and copy a k-contiguous operand (A when ta, B when not tb) element by element.
 template <typename T>
-int choose_variant(int64_t m, int64_t n, int64_t k, bool aligned, int64_t batch = 1) {
+int choose_variant(int64_t m, int64_t n, int64_t k, bool aligned, int64_t batch = 1, bool ta = false,
+                   bool tb = false) {
   const bool tma_ok = aligned && batch <= 1;
   const int count = variant_count_t<T>();
   TileChoice cand[16];
@@ -137,10 +140,20 @@ int choose_variant(int64_t m, int64_t n, int64_t k, bool aligned, int64_t batch 
     // weigh the more the smaller the tile (staging work per multiply-add goes with (BM+BN)/(BM*BN)); measured on
     // the 1001 x 999 x 1003 problem with odd leading dimensions.
     if (!aligned) eff *= 1.0 - 3.2 * (double)(vi.bm + vi.bn) / ((double)vi.bm * vi.bn);
+    // Element-wise transposing copies (FMA micro-kernels): the table's efficiency is measured in NN, where B is
+    // copied that way; the loss goes with the copied elements per multiply-add, 1/BN for A and 1/BM for B.
+    // Measured at 8192^3 (128 x 64 tile, TFLOP/s): NT 62.0, NN 57.9, TT 51.3, TN 47.6; 128 x 128: 63.7, 58.2, 56.8, 54.9.
+    if (strncmp(vi.micro, "ffma", 4) == 0 && sizeof(T) == 4) {
+      const double ca = 10.0, cb = 7.0;  // fitted to the eight figures above (within 3 %)
+      double f = (1.0 - (ta ? ca / vi.bn : 0.0) - (tb ? 0.0 : cb / vi.bm)) / (1.0 - cb / vi.bm);
+      if (f > 1.15) f = 1.15;  // the 32 x 32 tile gains 1.24-1.32 in NT, but the estimate already favours it at 1024^3
+      eff *= f;
+    }
     cand[v] = TileChoice{vi.bm, vi.bn, vi.bk, vi.threads, vi.ctas_per_sm, eff,
                          comparison_only || (needs_alignment && !tma_ok)};
     // measured: a TMA-staged CTA starts about 2 microseconds later than a cp.async one (512^3: 17.4 against 12.6 us)
     if (needs_alignment) cand[v].extra_fixed_clks = 4500.0;
+    cand[v].per_tile_extra_clks = vi.per_tile_extra_clks;
   }
   return select_tile(cand, count < 16 ? count : 16, m, n, k, sm_count_cached(), (int)sizeof(T), batch);
 }
@@ -155,7 +168,7 @@ int gemm_launch_checked(int variant, bool ta, bool tb, int64_t m, int64_t n, int
   constexpr int64_t kVec = 16 / (int64_t)sizeof(T);
   const bool aligned = operands_aligned(A, lda, B, ldb) &&
                        (ex.batch <= 1 || (ex.stride_a % kVec == 0 && ex.stride_b % kVec == 0));
-  if (variant == B2_VARIANT_AUTO) variant = choose_variant<T>(m, n, k, aligned, ex.batch);
+  if (variant == B2_VARIANT_AUTO) variant = choose_variant<T>(m, n, k, aligned, ex.batch, ta, tb);
   GemmArgs<T> args;
   args.m = m, args.n = n, args.k = k;
   args.alpha = alpha, args.beta = beta;
@@ -258,8 +271,9 @@ extern "C" int b2_gemm_query_config(int dtype, char transa, char transb, int64_t
   if (!json_out) return -11;
   const int elem = dtype == B2_F64 ? 8 : 4;
   const bool ld_aligned = (lda % (16 / elem) == 0) && (ldb % (16 / elem) == 0);
-  const int v = dtype == B2_F64 ? b2::choose_variant<double>(m, n, k, ld_aligned)
-                                : b2::choose_variant<float>(m, n, k, ld_aligned);
+  const bool ta = b2::is_t(transa), tb = b2::is_t(transb);
+  const int v = dtype == B2_F64 ? b2::choose_variant<double>(m, n, k, ld_aligned, 1, ta, tb)
+                                : b2::choose_variant<float>(m, n, k, ld_aligned, 1, ta, tb);
   const b2::VariantInfo& vi = dtype == B2_F64 ? b2::f64_variant_info(v) : b2::f32_variant_info(v);
   const long long tiles_m = (m + vi.bm - 1) / vi.bm, tiles_n = (n + vi.bn - 1) / vi.bn;
   char buf[768];

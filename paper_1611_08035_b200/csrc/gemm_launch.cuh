@@ -12,6 +12,8 @@ struct VariantInfo {
   const char* micro;  // "dmma" | "dfma" | "ffma"
   int bm, bn, bk, stages, threads, ctas_per_sm;
   double efficiency;  // measured steady-state fraction of the arithmetic pipe's peak (large interior problems)
+  int tm = 8, tn = 8;  // FMA micro-kernels: accumulator block per thread
+  double per_tile_extra_clks = 0.0;  // ramp-up and epilogue time of a tile that its co-resident CTAs do not cover
 };
 
 template <typename T>

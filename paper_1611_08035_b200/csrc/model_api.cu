@@ -36,9 +36,9 @@ extern "C" int b2_model_predict_variant(int dtype, int variant, double* fraction
   else if (strcmp(vi.micro, "ffma2") == 0) kind = MK_FFMA2;
   else kind = MK_FFMA;
   const int warps = vi.threads / 32;
-  // warp tile: DMMA variants split the CTA tile 2 x (warps/2); FMA variants always use 64 x 32 per warp
-  const int wtm = kind == MK_DMMA ? vi.bm / 2 : 64;
-  const int wtn = kind == MK_DMMA ? vi.bn / (warps / 2) : 32;
+  // warp tile: DMMA variants split the CTA tile 2 x (warps/2); FMA variants cover 8 x 4 lanes of tm x tn blocks
+  const int wtm = kind == MK_DMMA ? vi.bm / 2 : 8 * vi.tm;
+  const int wtn = kind == MK_DMMA ? vi.bn / (warps / 2) : 4 * vi.tn;
   const int elem = dtype == B2_F64 ? 8 : 4;
   const int staging = (vi.bm + vi.bn) * vi.bk * elem / 16 / vi.threads;  // 16-byte chunks per thread per slab
   const WarpMix mix = warp_mix(kind, wtm, wtn, staging, vi.bk);

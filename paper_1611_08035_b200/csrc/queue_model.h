@@ -63,7 +63,8 @@ inline void sm_rates(double (&rate)[NPIPES]) {
 enum MicroKind { MK_DMMA = 0, MK_DFMA = 1, MK_FFMA = 2, MK_FFMA2 = 3 };
 
 // Jobs per pipeline for one rank-1 update (one k) of one warp's tile.
-//   wtm x wtn     the warp's block of C (DMMA: 16x8 fragments; FMA kinds: 8 lanes x 4 lanes of 8x8 blocks = 64x32)
+//   wtm x wtn     the warp's block of C (DMMA: 16x8 fragments; FMA kinds: 8 lanes x 4 lanes of tm x tn blocks,
+//                 8 x 8 -> 64 x 32, 16 x 8 -> 128 x 32, 4 x 4 -> 32 x 16)
 //   staging       cp.async instructions per thread per slab, slab_k = BK
 struct WarpMix {
   double jobs[NPIPES];
@@ -82,9 +83,10 @@ inline WarpMix warp_mix(int kind, int wtm, int wtn, int staging_per_slab, int sl
     m.jobs[LSU] = (mi * 4.0 + ni * 2.0) / 4.0;   // 512 and 256 distinct bytes per warp load
     m.jobs[ISSUE] = mi * ni / 4.0 + loads + overhead;
   } else {
-    const double fma = 64.0;                     // 8 x 8 block per lane
+    const double tm = wtm / 8.0, tn = wtn / 4.0;  // accumulator block per lane
+    const double fma = tm * tn;
     const bool f64 = (kind == MK_DFMA);
-    const double loads = f64 ? 8.0 : 4.0;        // 16 operand values per lane in 16-byte loads
+    const double loads = (tm + tn) / (f64 ? 2.0 : 4.0);  // tm + tn operand values per lane in 16-byte loads
     m.jobs[LSU] = loads;                         // lanes of a warp share operands: one wavefront per load
     if (kind == MK_DFMA) {
       m.jobs[FP64] = fma;
@@ -94,7 +96,7 @@ inline WarpMix warp_mix(int kind, int wtm, int wtn, int staging_per_slab, int sl
       m.jobs[ISSUE] = fma + loads + overhead;
     } else {
       m.jobs[FP32] = fma;                        // 32 packed instructions, two jobs each
-      m.jobs[ISSUE] = fma / 2.0 + loads + 8.0 + overhead;  // plus eight moves that duplicate b
+      m.jobs[ISSUE] = fma / 2.0 + loads + tn + overhead;  // plus the moves that duplicate the tn values of b
     }
   }
   return m;

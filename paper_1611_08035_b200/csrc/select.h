@@ -19,6 +19,7 @@ struct TileChoice {
   double efficiency;  // measured steady-state fraction of the arithmetic pipe's peak
   bool explicit_only;  // never chosen automatically (comparison variants)
   double extra_fixed_clks = 0.0;  // start-up cost beyond the common one (TMA: descriptor fetch, barrier set-up)
+  double per_tile_extra_clks = 0.0;  // exposed ramp-up/epilogue time per tile (variants with few, large CTAs per SM)
 };
 
 // Measured / derived machine rates per SM (B200): FP64 and FP32 multiply-adds per clock, the
@@ -69,7 +70,7 @@ inline double estimate_clks(const TileChoice& c, int64_t m, int64_t n, int64_t k
   auto tile_clks = [&](double occ) {
     const double t_math = fma_tile / (r.fma_per_clk * c.efficiency * occ);
     const double t_main = t_math > t_feed ? t_math : t_feed;
-    return t_main > t_epi ? t_main : t_epi;
+    return (t_main > t_epi ? t_main : t_epi) + c.per_tile_extra_clks;
   };
   if (per_sm < 2.0) return per_sm * (tile_clks(occupancy(1.0)) + t_fixed);  // nothing overlaps the fixed costs
   double total = full_groups * cps * tile_clks(1.0);
