@@ -30,7 +30,8 @@ constexpr int TBM = 128, TBK = 32, UMMA_K = 8;
 constexpr uint32_t STAGE_A_BYTES = TBM * TBK * 4;
 // Tile width (TBN) and ring depth: 128 x 256 tiles with 4 stages halve the shared-memory bytes read per
 // multiply-add (the tensor pipe reads A and B from shared memory for every instruction); 128 x 128 tiles with 6
-// stages serve narrow problems.  Either ring is 192 KB.
+// stages serve narrow problems.  Either ring is 192 KB; the 2-stage ring of the 128 x 256 tile (96 KB) lets two
+// CTAs share an SM.
 template <int TBN, int TSTAGES>
 struct Tf32Cfg {
   static constexpr uint32_t STAGE_B_BYTES = TBN * TBK * 4;
@@ -137,18 +138,25 @@ __device__ __forceinline__ void umma_commit(uint64_t* bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
                : "memory");
 }
-// 16 consecutive accumulator columns of this lane's row (32 lanes x 32 bits, 16 repetitions).
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16]) {
-  uint32_t r[16];
+// 16 consecutive accumulator columns of this lane's row (32 lanes x 32 bits, 16 repetitions); the values are
+// defined only after tmem_ld_wait().
+__device__ __forceinline__ void tmem_ld16_issue(uint32_t taddr, uint32_t (&r)[16]) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
       : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
         "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
       : "r"(taddr)
       : "memory");
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+// The registers pass through the wait as read-write operands, so that no use of them is scheduled before it.
+__device__ __forceinline__ void tmem_ld_wait(uint32_t (&a)[16], uint32_t (&b)[16]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+r"(a[0]), "+r"(a[1]), "+r"(a[2]), "+r"(a[3]), "+r"(a[4]), "+r"(a[5]), "+r"(a[6]), "+r"(a[7]),
+                 "+r"(a[8]), "+r"(a[9]), "+r"(a[10]), "+r"(a[11]), "+r"(a[12]), "+r"(a[13]), "+r"(a[14]), "+r"(a[15]),
+                 "+r"(b[0]), "+r"(b[1]), "+r"(b[2]), "+r"(b[3]), "+r"(b[4]), "+r"(b[5]), "+r"(b[6]), "+r"(b[7]),
+                 "+r"(b[8]), "+r"(b[9]), "+r"(b[10]), "+r"(b[11]), "+r"(b[12]), "+r"(b[13]), "+r"(b[14]), "+r"(b[15])
+               :
+               : "memory");
 }
 
 // Shared-memory matrix descriptor of a K-major operand tile stored as rows of 128 bytes (32 floats) with the
@@ -179,8 +187,8 @@ struct Tf32Args {
   int* status;
 };
 
-template <int TBN, int TSTAGES>
-__global__ void __launch_bounds__(128, 1)
+template <int TBN, int TSTAGES, int MINB = 1>
+__global__ void __launch_bounds__(128, MINB)
     sgemm_tf32_kernel(const Tf32Args p, const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB) {
   constexpr uint32_t STAGE_B_BYTES = Tf32Cfg<TBN, TSTAGES>::STAGE_B_BYTES;
   constexpr uint32_t RING_BYTES = Tf32Cfg<TBN, TSTAGES>::RING_BYTES;
@@ -272,22 +280,27 @@ __global__ void __launch_bounds__(128, 1)
       const int64_t row = m0 + warp * 32 + lane;
       const uint32_t taddr = tmem_d + ((uint32_t)(warp * 32) << 16);
       const bool use_beta = (p.beta != 0.0f);
-      for (int c0 = 0; c0 < TBN; c0 += 16) {
-        float v[16], old[16];
-        tmem_ld16(taddr + (uint32_t)c0, v);  // all lanes take part (the load is warp-wide)
-        if (row < p.m) {
-          if (use_beta) {
+      // 32 columns per step: the old C values are requested first, so that their latency runs under the
+      // accumulator load; both are complete before the first store.
+      for (int c0 = 0; c0 < TBN; c0 += 32) {
+        float old[32];
+        if (use_beta && row < p.m) {
 #pragma unroll
-            for (int j = 0; j < 16; ++j) {
-              const int64_t col = n0 + c0 + j;
-              old[j] = (col < p.n) ? p.C[row + col * p.ldc] : 0.0f;
-            }
+          for (int j = 0; j < 32; ++j) {
+            const int64_t col = n0 + c0 + j;
+            old[j] = (col < p.n) ? p.C[row + col * p.ldc] : 0.0f;
           }
+        }
+        uint32_t r0[16], r1[16];
+        tmem_ld16_issue(taddr + (uint32_t)c0, r0);  // all lanes take part (the loads are warp-wide)
+        tmem_ld16_issue(taddr + (uint32_t)c0 + 16u, r1);
+        tmem_ld_wait(r0, r1);
+        if (row < p.m) {
 #pragma unroll
-          for (int j = 0; j < 16; ++j) {
+          for (int j = 0; j < 32; ++j) {
             const int64_t col = n0 + c0 + j;
             if (col < p.n) {
-              float out = p.alpha * v[j];
+              float out = p.alpha * __uint_as_float(j < 16 ? r0[j] : r1[j - 16]);
               if (use_beta) out += p.beta * old[j];
               p.C[row + col * p.ldc] = out;
             }
@@ -337,10 +350,10 @@ bool panel_map(CUtensorMap* map, const float* P, int64_t rows, int64_t pitch, in
 
 bool t_is_n(char c) { return c == 'N' || c == 'n'; }
 
-template <int TBN, int TSTAGES>
+template <int TBN, int TSTAGES, int MINB = 1>
 int launch_tf32(const Tf32Args& a, const float* PA, const float* PB, int64_t pitch, int dev, cudaStream_t st) {
   static bool configured[64] = {};
-  auto kfn = sgemm_tf32_kernel<TBN, TSTAGES>;
+  auto kfn = sgemm_tf32_kernel<TBN, TSTAGES, MINB>;
   constexpr size_t smem = Tf32Cfg<TBN, TSTAGES>::SMEM_BYTES;
   if (!configured[dev]) {
     if (cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
@@ -414,7 +427,20 @@ int sgemm_tf32(int terms, char transa, char transb, int64_t m, int64_t n, int64_
   a.status = status_by_device[dev];
   // wide tiles unless they would leave SMs without work that narrow tiles can fill
   const long long wide_tiles = (long long)a.tiles_m * ((n + 255) / 256);
-  if (n > 128 && wide_tiles >= 96) return launch_tf32<256, 4>(a, PA, PB, pl.pitch, dev, st);
+  if (n > 128 && wide_tiles >= 96) {
+    // More than one wave of tiles and a main loop short enough for the epilogue to matter: two CTAs per SM, each
+    // with a 2-stage ring (96 KB) and 256 of the 512 tensor-memory columns, so that one CTA's epilogue and ramp-up
+    // run under the other's multiply-adds.  Measured (TFLOP/s, packing included, against one CTA with 4 stages):
+    // 3072^3 440 / 386, 4096^3 476 / 412, 8192^3 663 / 592, three-term 4096^3 200 / 187, 8192^3 225 / 228.
+    static int sms_by_device[64] = {};
+    if (sms_by_device[dev] == 0) {
+      int sms = 0;
+      if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) sms = 148;
+      sms_by_device[dev] = sms;
+    }
+    if (wide_tiles > sms_by_device[dev] && a.kt <= 512) return launch_tf32<256, 2, 2>(a, PA, PB, pl.pitch, dev, st);
+    return launch_tf32<256, 4>(a, PA, PB, pl.pitch, dev, st);
+  }
   return launch_tf32<128, 6>(a, PA, PB, pl.pitch, dev, st);
 }
 
