@@ -196,6 +196,10 @@ def other_configs(b2, device):
         real("d", "N", "N", s, s, s, 1.5, 0.5, "uniform", 2000, False, f"dgemm_nn_{s}")
     for s in (512, 1024, 2048, 4096, 8192):
         real("s", "N", "N", s, s, s, 1.5, 0.5, "uniform", 2100, False, f"sgemm_nn_{s}")
+    for kind in "ds":  # the other three transpose combinations of the 4096^3 problem
+        for ta, tb in (("N", "T"), ("T", "N"), ("T", "T")):
+            real(kind, ta, tb, 4096, 4096, 4096, 1.5, 0.5, "uniform", 2200, False,
+                 f"{kind}gemm_{ta.lower()}{tb.lower()}_4096")
     for k in (64, 128, 256):
         real("d", "N", "N", 16384, 16384, k, -1.0, 1.0, "normal", 3000 + k, False, f"rank_k_dgemm_16384_k{k}")
     for kind in "ds":
