@@ -80,6 +80,15 @@ def test_tf32_large_sampled(b2, oracle, terms):
     run_tf32(b2, oracle, terms, "N", "N", size, size, size, 1.5, 0.5, dist="int9", seed=2100, cols=cols, expect_exact=True)
 
 
+@pytest.mark.parametrize("terms", [1, 3])
+def test_tf32_ragged_wide_tiles_both_residencies(b2, oracle, terms):
+    """128 x 256 tiles with ragged last tile rows and columns, in both launch forms: 12 x 12 = 144 tiles (one wave,
+    one CTA per SM with the 4-stage ring) and 16 x 13 = 208 tiles (more than one wave: two CTAs per SM, 2-stage rings)."""
+    run_tf32(b2, oracle, terms, "N", "T", 1500, 3000, 100, 0.7, -0.3, seed=31)
+    run_tf32(b2, oracle, terms, "T", "N", 2000, 3100, 70, 1.5, 0.5, dist="int9", seed=32, expect_exact=True)
+    run_tf32(b2, oracle, terms, "N", "N", 2000, 3100, 70, 0.7, -0.3, seed=33, pad=True)
+
+
 def test_tf32_quick_returns_and_errors(b2):
     m, n, k = 40, 30, 20
     A, lda, B, ldb, C, ldc = synth.gemm_inputs("N", "N", m, n, k, "uniform", 5, torch.float32)
