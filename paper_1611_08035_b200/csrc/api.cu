@@ -44,8 +44,8 @@ const LaunchFn<double> kF64Launch[] = {launch_f64_v0, launch_f64_v1, launch_f64_
                                        launch_f64_v4, launch_f64_v5, launch_f64_v6, launch_f64_t32,
                                        launch_f64_tma_t32};
 const VariantInfo kF32Info[] = {
-    {"ffma2_t16x8_128x128x16_s3", "ffma2", 128, 128, 16, 3, 128, 2, 0.78, 16, 8, 3500.0},
-    {"ffma2_128x64x16_s4", "ffma2", 128, 64, 16, 4, 128, 3, 0.775},
+    {"ffma2_t16x8_128x128x16_s3", "ffma2", 128, 128, 16, 3, 128, 2, 0.782, 16, 8, 3500.0, 11.0},
+    {"ffma2_128x64x16_s4", "ffma2", 128, 64, 16, 4, 128, 3, 0.795, 8, 8, 0.0, 5.8},
     {"ffma2_64x64x16_s4", "ffma2", 64, 64, 16, 4, 64, 6, 0.64},
     {"ffma_128x64x16_s4", "ffma", 128, 64, 16, 4, 128, 4, 0.70},
     {"ffma2_t4_32x32x16_s4", "ffma2", 32, 32, 16, 4, 64, 8, 0.40, 4, 4},
@@ -142,9 +142,10 @@ int choose_variant(int64_t m, int64_t n, int64_t k, bool aligned, int64_t batch 
     if (!aligned) eff *= 1.0 - 3.2 * (double)(vi.bm + vi.bn) / ((double)vi.bm * vi.bn);
     // Element-wise transposing copies (FMA micro-kernels): the table's efficiency is measured in NN, where B is
     // copied that way; the loss goes with the copied elements per multiply-add, 1/BN for A and 1/BM for B.
-    // Measured at 8192^3 (128 x 64 tile, TFLOP/s): NT 62.0, NN 57.9, TT 51.3, TN 47.6; 128 x 128: 63.7, 58.2, 56.8, 54.9.
+    // Measured at 8192^3 (128 x 64 tile, TFLOP/s): NT 62.0, NN 59.2, TT 51.3, TN 47.1; 128 x 128: 63.7, 58.2, 56.8, 54.9.
+    // The cost of B's copy differs per variant (128 x 64 transposes it through registers).
     if (strncmp(vi.micro, "ffma", 4) == 0 && sizeof(T) == 4) {
-      const double ca = 10.0, cb = 7.0;  // fitted to the eight figures above (within 3 %)
+      const double ca = 10.0, cb = vi.transpose_b_cost;  // fitted to the eight figures above (within 4 %)
       double f = (1.0 - (ta ? ca / vi.bn : 0.0) - (tb ? 0.0 : cb / vi.bm)) / (1.0 - cb / vi.bm);
       if (f > 1.15) f = 1.15;  // the 32 x 32 tile gains 1.24-1.32 in NT, but the estimate already favours it at 1024^3
       eff *= f;

@@ -182,6 +182,7 @@ struct DmmaMicro {
   static constexpr int NT = 32 * WARPS_M * WARPS_N;
   static constexpr int WTM = BM / WARPS_M, WTN = BN / WARPS_N;
   static constexpr int MI = WTM / 16, NI = WTN / 8;
+  static constexpr bool REG_TRANSPOSE_B = false;
   static_assert(WTM % 16 == 0 && WTN % 8 == 0 && BK % 16 == 0, "warp tile must be built from 16x8 fragments");
   // Fragment loads read either layout, so tiles are staged in their source layout.
   static constexpr Layout LA = TA ? KC : OC;
@@ -340,8 +341,11 @@ struct DmmaMicro {
 // A warp is 8 lanes along m by 4 lanes along n, so it covers 64 x 32 of C.
 // ---------------------------------------------------------------------------------------
 template <typename T_, int BM_, int BN_, int BK_, int WARPS_M, int WARPS_N, bool TA, bool TB, bool PACKED = true,
-          int TM_ = 8, int TN_ = 8>
+          int TM_ = 8, int TN_ = 8, bool REGB_ = false>
 struct SimtMicro {
+  // REGB: a k-contiguous B (not transposed) is transposed through registers (16-byte global loads along k, 4-byte
+  // shared-memory stores) instead of by 4-byte cp.async; see GemmKernel::run.
+  static constexpr bool REG_TRANSPOSE_B = REGB_ && !TB && sizeof(T_) == 4;
   using T = T_;
   // fp32 only: PACKED uses the pair instruction fma.rn.f32x2; false keeps scalar FFMA (comparison variant)
   static constexpr bool PAIRS = (sizeof(T_) == 4) && PACKED;
@@ -634,14 +638,61 @@ struct GemmKernel {
     typename Micro::Acc acc;
     Micro::zero(acc);
 
+    // Transposition of a k-contiguous B through registers (fp32 FMA kernels, 16-byte aligned columns, full
+    // interior slabs): while slab kt is being multiplied, the thread's share of slab kt+STAGES-1 travels from
+    // global memory into registers in 16-byte pieces along k; after the multiply-adds it is written to the free
+    // ring slot element by element, transposed.  A pair of lanes reads one 32-byte sector of a column, a warp 16
+    // columns; the stores of a warp fall into 32 different banks (pitch = 4 mod 32 words).  The next CTA-wide
+    // barrier publishes the slot, which is not read before the iteration after it.
+    constexpr bool REGB = Micro::REG_TRANSPOSE_B && ALIGNED;
+    constexpr int NBR = REGB ? (BN * BK / 4) / NT : 1;
+    static_assert(!REGB || ((BN * BK / 4) % NT == 0 && (BK / 4) % 2 == 0 && NT % 2 == 0 && (BN % (NT / 2) == 0 || (NT / 2) % BN == 0)),
+                  "register transposition geometry");
+    float4 breg[NBR];
+
     // steady state: wait for slab kt, refill the slot freed in the previous iteration, compute
     int slot = 0, fill = STAGES - 1;
     for (int kt = 0; kt < KT; ++kt) {
       cp_async_wait<STAGES - 2>();
       __syncthreads();
-      if (kt + STAGES - 1 < KT) stage(kt + STAGES - 1, fill);
+      const int next = kt + STAGES - 1;
+      bool by_regs = false;
+      if constexpr (REGB) by_regs = (next < KT) && b_inside && (next != KT - 1 || k_tail == BK);
+      if (by_regs) {
+        if constexpr (REGB) {
+          T* dA = sA + fill * Micro::A_STAGE;
+          if (a_inside) {
+            stA.load_fast(dA, p.lda, tid);
+          } else {
+            stA.load_edge(dA, p.lda, m_valid, tid);
+          }
+          stA.advance(p.lda);
+          stB.advance(p.ldb);
+          const T* gBn = gB + (int64_t)next * BK;
+#pragma unroll
+          for (int it = 0; it < NBR; ++it) {
+            const int c = tid + it * NT;
+            const int n = (c >> 1) % BN, kq = ((c >> 1) / BN) * 2 + (c & 1);
+            breg[it] = *reinterpret_cast<const float4*>(gBn + (int64_t)n * p.ldb + kq * 4);
+          }
+        }
+      } else if (next < KT) {
+        stage(next, fill);
+      }
       cp_async_commit();
       Micro::compute(acc, sA + slot * Micro::A_STAGE, sB + slot * Micro::B_STAGE, warp_m, warp_n, lane);
+      if constexpr (REGB) {
+        if (by_regs) {
+          T* dB = sB + fill * Micro::B_STAGE;
+#pragma unroll
+          for (int it = 0; it < NBR; ++it) {
+            const int c = tid + it * NT;
+            const int n = (c >> 1) % BN, kq = ((c >> 1) / BN) * 2 + (c & 1);
+            T* d = dB + (kq * 4) * Micro::PB + n;
+            d[0] = breg[it].x, d[Micro::PB] = breg[it].y, d[2 * Micro::PB] = breg[it].z, d[3 * Micro::PB] = breg[it].w;
+          }
+        }
+      }
       slot = (slot + 1 == STAGES) ? 0 : slot + 1;
       fill = (fill + 1 == STAGES) ? 0 : fill + 1;
     }

@@ -14,6 +14,7 @@ struct VariantInfo {
   double efficiency;  // measured steady-state fraction of the arithmetic pipe's peak (large interior problems)
   int tm = 8, tn = 8;  // FMA micro-kernels: accumulator block per thread
   double per_tile_extra_clks = 0.0;  // ramp-up and epilogue time of a tile that its co-resident CTAs do not cover
+  double transpose_b_cost = 7.0;     // FMA micro-kernels: loss to the transposing copy of a k-contiguous B is cost/BM
 };
 
 template <typename T>
