@@ -89,6 +89,18 @@ def test_tf32_ragged_wide_tiles_both_residencies(b2, oracle, terms):
     run_tf32(b2, oracle, terms, "N", "N", 2000, 3100, 70, 0.7, -0.3, seed=33, pad=True)
 
 
+def test_tf32_long_k_several_waves(b2, oracle):
+    """More than 512 k-slabs and more than one wave of ragged 128 x 256 tiles: the launch form with one CTA per SM
+    and the 4-stage ring, whose slots and barrier phases wrap many times (beta != 0 and integer data)."""
+    m, n, k = 2000, 3100, 5500   # three-term: 516 slabs, 16 x 13 = 208 tiles on 148 CTAs
+    cols = sample_columns(n, tile=256, extra=8, seed=5)
+    run_tf32(b2, oracle, 3, "N", "N", m, n, k, 0.7, -0.3, seed=41, cols=cols)
+    run_tf32(b2, oracle, 3, "T", "T", m, n, k, 1.5, 0.5, dist="int9", seed=42, cols=cols, expect_exact=True)
+    m, n, k = 2500, 5000, 16500  # one-term: 516 slabs, 20 x 20 = 400 tiles
+    cols = sample_columns(n, tile=256, extra=4, seed=6)
+    run_tf32(b2, oracle, 1, "N", "T", m, n, k, 1.5, 0.5, dist="int9", seed=43, cols=cols, expect_exact=True)
+
+
 def test_tf32_quick_returns_and_errors(b2):
     m, n, k = 40, 30, 20
     A, lda, B, ldb, C, ldc = synth.gemm_inputs("N", "N", m, n, k, "uniform", 5, torch.float32)
