@@ -431,7 +431,11 @@ def main():
                        "layout": "column-major NN, lda=ldb=ldc=8192", "kernel": cfg["name"],
                        "l2": "operands (3 x 512 MiB) are larger than the 126 MB L2; no flush between steps",
                        "multi_gpu": "independent replicas, one problem per GPU, no collective"},
+            "ms_per_step_median": statistics.median(per_step), "ms_per_step_min": min(per_step),
             "frac_of_fp64_peak": value / world / 1e3 / FP64_PEAK_TFLOPS,
+            "frac_of_fp64_peak_at_observed_clock": (
+                value / world / 1e3 / (FP64_PEAK_TFLOPS * clocks["sm_mhz"] / 1965.0)
+                if clocks and clocks.get("sm_mhz") else None),
             "fp64_peak_tflops": FP64_PEAK_TFLOPS,
             "fp64_peak_source": "148 SMs x 64 FP64 FMA/clk/SM (measured by the DFMA and DMMA probes) x 2 x 1.965 GHz",
             "clocks": clocks,
