@@ -45,7 +45,7 @@ const LaunchFn<double> kF64Launch[] = {launch_f64_v0, launch_f64_v1, launch_f64_
                                        launch_f64_tma_t32};
 const VariantInfo kF32Info[] = {
     {"ffma2_t16x8_128x128x16_s3", "ffma2", 128, 128, 16, 3, 128, 2, 0.782, 16, 8, 3500.0, 11.0},
-    {"ffma2_128x64x16_s4", "ffma2", 128, 64, 16, 4, 128, 3, 0.795, 8, 8, 0.0, 5.8},
+    {"ffma2_128x64x16_s4", "ffma2", 128, 64, 16, 4, 128, 3, 0.795, 8, 8, 0.0, 5.8, true},
     {"ffma2_64x64x16_s4", "ffma2", 64, 64, 16, 4, 64, 6, 0.64},
     {"ffma_128x64x16_s4", "ffma", 128, 64, 16, 4, 128, 4, 0.70},
     {"ffma2_t4_32x32x16_s4", "ffma2", 32, 32, 16, 4, 64, 8, 0.40, 4, 4},
@@ -125,9 +125,14 @@ static bool operands_aligned(const T* A, int64_t lda, const T* B, int64_t ldb) {
 // single problem (`batch` <= 1).
 // ta / tb: op(A) = A^T, op(B) = B^T.  They matter to the FMA micro-kernels only, which want both operands packed
 // with the C index contiguous and copy a k-contiguous operand (A when ta, B when not tb) element by element.
+// ksplit_out (optional): where a variant can split the k-loop of a tile over a cluster of 2 or 4 CTAs, the same
+// estimate is made for the problem seen as 2 or 4 times the tiles with a half or a quarter of k, plus what the
+// reduction costs a tile; the best (variant, split) pair wins.  Measured with the 128 x 64 fp32 tile (us, split 1 /
+// 2 / 4): 768^3 45.1 / 28.7 / 36.9, 1024^3 57.9 / 53.7 / 58.0, 1536^3 141 / 142 / 162, 2048^3 355 / 312 / 343,
+// 3072^3 1031 / 1031 / 1086.
 template <typename T>
 int choose_variant(int64_t m, int64_t n, int64_t k, bool aligned, int64_t batch = 1, bool ta = false,
-                   bool tb = false) {
+                   bool tb = false, int* ksplit_out = nullptr) {
   const bool tma_ok = aligned && batch <= 1;
   const int count = variant_count_t<T>();
   TileChoice cand[16];
@@ -156,7 +161,31 @@ int choose_variant(int64_t m, int64_t n, int64_t k, bool aligned, int64_t batch 
     if (needs_alignment) cand[v].extra_fixed_clks = 4500.0;
     cand[v].per_tile_extra_clks = vi.per_tile_extra_clks;
   }
-  return select_tile(cand, count < 16 ? count : 16, m, n, k, sm_count_cached(), (int)sizeof(T), batch);
+  const int sms = sm_count_cached();
+  int best = select_tile(cand, count < 16 ? count : 16, m, n, k, sms, (int)sizeof(T), batch);
+  if (ksplit_out) {
+    *ksplit_out = 1;
+    double best_t = estimate_clks(cand[best], m, n, k, sms, (int)sizeof(T), batch);
+    for (int v = 0; v < count && v < 16; ++v) {
+      const VariantInfo& vi = variant_info_t<T>(v);
+      if (!vi.can_ksplit || cand[v].explicit_only) continue;
+      for (int split = 2; split <= 2; split *= 2) {  // 4 CTAs per tile never beat the better of 1 and 2 where measured
+        const int64_t slabs = (k + vi.bk - 1) / vi.bk;
+        if (slabs < 8 * split) break;  // keep at least 8 slabs per CTA
+        // with fewer tiles than a quarter of the SMs the 32 x 32 tile is the better tool (512^3 TN: 18.5 us against 24.4)
+        const int64_t tiles = ((m + vi.bm - 1) / vi.bm) * ((n + vi.bn - 1) / vi.bn) * (batch < 1 ? 1 : batch);
+        if (4 * tiles < sms) break;
+        const int64_t k_part = (slabs + split - 1) / split * vi.bk;
+        TileChoice c = cand[v];
+        // reduction: two cluster barriers and, for the first CTA, the other CTAs' accumulators through
+        // distributed shared memory
+        c.per_tile_extra_clks += 1500.0 + (split - 1) * (double)vi.bm * vi.bn * sizeof(T) / 32.0 / split;
+        const double t = estimate_clks(c, m, n, k_part, sms, (int)sizeof(T), batch * split);
+        if (t < 0.97 * best_t) best = v, best_t = t, *ksplit_out = split;  // a split has to win by 3 %
+      }
+    }
+  }
+  return best;
 }
 
 // Variant choice and launch of an already checked, non-trivial problem (m, n, k > 0, alpha != 0).
@@ -169,12 +198,15 @@ int gemm_launch_checked(int variant, bool ta, bool tb, int64_t m, int64_t n, int
   constexpr int64_t kVec = 16 / (int64_t)sizeof(T);
   const bool aligned = operands_aligned(A, lda, B, ldb) &&
                        (ex.batch <= 1 || (ex.stride_a % kVec == 0 && ex.stride_b % kVec == 0));
-  if (variant == B2_VARIANT_AUTO) variant = choose_variant<T>(m, n, k, aligned, ex.batch, ta, tb);
+  int ksplit = 1;
+  if (variant == B2_VARIANT_AUTO)
+    variant = choose_variant<T>(m, n, k, aligned, ex.batch, ta, tb, ex.tri == 0 ? &ksplit : nullptr);
   GemmArgs<T> args;
   args.m = m, args.n = n, args.k = k;
   args.alpha = alpha, args.beta = beta;
   args.A = A, args.lda = lda, args.B = B, args.ldb = ldb, args.C = C, args.ldc = ldc;
   args.tiles_m = args.tiles_n = 0;
+  args.ksplit = ksplit;
   args.tri = ex.tri;
   args.batch = ex.batch, args.batch_a = ex.stride_a, args.batch_b = ex.stride_b, args.batch_c = ex.stride_c;
   // Rasterisation group: the CTAs resident at one time should cover a block of C whose A row-panels and
@@ -273,8 +305,9 @@ extern "C" int b2_gemm_query_config(int dtype, char transa, char transb, int64_t
   const int elem = dtype == B2_F64 ? 8 : 4;
   const bool ld_aligned = (lda % (16 / elem) == 0) && (ldb % (16 / elem) == 0);
   const bool ta = b2::is_t(transa), tb = b2::is_t(transb);
-  const int v = dtype == B2_F64 ? b2::choose_variant<double>(m, n, k, ld_aligned, 1, ta, tb)
-                                : b2::choose_variant<float>(m, n, k, ld_aligned, 1, ta, tb);
+  int ksplit = 1;
+  const int v = dtype == B2_F64 ? b2::choose_variant<double>(m, n, k, ld_aligned, 1, ta, tb, &ksplit)
+                                : b2::choose_variant<float>(m, n, k, ld_aligned, 1, ta, tb, &ksplit);
   const b2::VariantInfo& vi = dtype == B2_F64 ? b2::f64_variant_info(v) : b2::f32_variant_info(v);
   const long long tiles_m = (m + vi.bm - 1) / vi.bm, tiles_n = (n + vi.bn - 1) / vi.bn;
   char buf[768];
@@ -282,9 +315,9 @@ extern "C" int b2_gemm_query_config(int dtype, char transa, char transb, int64_t
       buf, sizeof(buf),
       "{\"dtype\": \"%s\", \"variant\": %d, \"name\": \"%s\", \"micro_kernel\": \"%s\", \"BM\": %d, \"BN\": %d, "
       "\"kc\": %d, \"stages\": %d, \"threads\": %d, \"ctas_per_sm\": %d, \"grid\": %lld, \"tiles_m\": %lld, "
-      "\"tiles_n\": %lld, \"k_slabs\": %lld, \"vector_staging_if_pointers_aligned\": %s, \"sm_count\": %d}",
+      "\"tiles_n\": %lld, \"k_slabs\": %lld, \"k_split\": %d, \"vector_staging_if_pointers_aligned\": %s, \"sm_count\": %d}",
       dtype == B2_F64 ? "f64" : "f32", v, vi.name, vi.micro, vi.bm, vi.bn, vi.bk, vi.stages, vi.threads,
-      vi.ctas_per_sm, tiles_m * tiles_n, tiles_m, tiles_n, (long long)((k + vi.bk - 1) / vi.bk),
+      vi.ctas_per_sm, tiles_m * tiles_n * ksplit, tiles_m, tiles_n, (long long)((k + vi.bk - 1) / vi.bk), ksplit,
       ld_aligned ? "true" : "false", b2::sm_count_cached());
   if (len < 0 || (size_t)len + 1 > cap) return B2_ERR_WORKSPACE;
   memcpy(json_out, buf, (size_t)len + 1);

@@ -21,8 +21,30 @@ struct GemmArgs {
   int group_m;           // rasterisation: tile rows per group
   int tri;               // 0: all of C;  1: only i >= j (lower triangle);  2: only i <= j (upper triangle)
   int batch;             // number of problems of a strided batch (grid.y), at most 65535 per launch
+  // k split over a thread-block cluster (grid.z = cluster size = ksplit, 1: off): CTA z of a cluster multiplies
+  // the z-th share of the k-slabs of its tile; the shares are summed in rank order by CTA 0 through
+  // distributed shared memory, which then runs the epilogue.
+  int ksplit;
   int64_t batch_a, batch_b, batch_c;  // element offsets between the operands of consecutive problems
 };
+
+// ---- thread-block cluster helpers ---------------------------------------------------------
+// All threads of all CTAs of the cluster arrive and wait (no thread of a split launch leaves before both
+// barriers of the reduction, so the barrier always completes).
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// Address of `local_smem_addr` (a shared::cta address) in the shared memory of CTA `rank` of the cluster.
+__device__ __forceinline__ uint32_t cluster_map_shared(uint32_t local_smem_addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_smem_addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ unsigned long long ld_cluster_b64(uint32_t addr) {
+  unsigned long long v;
+  asm volatile("ld.shared::cluster.b64 %0, [%1];" : "=l"(v) : "r"(addr) : "memory");
+  return v;
+}
 
 // Does the BM x BN tile at (m0, n0) lie entirely outside the stored triangle?
 __device__ __forceinline__ bool tile_outside_triangle(int tri, int64_t m0, int64_t n0, int bm, int bn) {

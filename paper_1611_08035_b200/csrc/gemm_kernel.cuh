@@ -183,6 +183,7 @@ struct DmmaMicro {
   static constexpr int WTM = BM / WARPS_M, WTN = BN / WARPS_N;
   static constexpr int MI = WTM / 16, NI = WTN / 8;
   static constexpr bool REG_TRANSPOSE_B = false;
+  static constexpr bool HAS_KSPLIT = false;
   static_assert(WTM % 16 == 0 && WTN % 8 == 0 && BK % 16 == 0, "warp tile must be built from 16x8 fragments");
   // Fragment loads read either layout, so tiles are staged in their source layout.
   static constexpr Layout LA = TA ? KC : OC;
@@ -346,6 +347,9 @@ struct SimtMicro {
   // REGB: a k-contiguous B (not transposed) is transposed through registers (16-byte global loads along k, 4-byte
   // shared-memory stores) instead of by 4-byte cp.async; see GemmKernel::run.
   static constexpr bool REG_TRANSPOSE_B = REGB_ && !TB && sizeof(T_) == 4;
+  // k split over a cluster (fp32 packed-pair kernels): the accumulators of a thread as TM/2 * TN 64-bit words
+  static constexpr bool HAS_KSPLIT = (sizeof(T_) == 4) && PACKED;
+  static constexpr int ACC_WORDS = (TM_ / 2) * TN_;
   using T = T_;
   // fp32 only: PACKED uses the pair instruction fma.rn.f32x2; false keeps scalar FFMA (comparison variant)
   static constexpr bool PAIRS = (sizeof(T_) == 4) && PACKED;
@@ -370,6 +374,15 @@ struct SimtMicro {
     unsigned long long p[TM / 2][TN];
   };
   using Acc = typename std::conditional<PAIRS, AccPairs, AccScalar>::type;
+  static __device__ __forceinline__ unsigned long long& word(AccPairs& acc, int w) { return acc.p[w / TN][w % TN]; }
+  // a += b on both halves of a pair (two IEEE fp32 additions)
+  static __device__ __forceinline__ void add_pair(unsigned long long& a, unsigned long long b) {
+    float a0, a1, b0, b1;
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(a0), "=f"(a1) : "l"(a));
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(b0), "=f"(b1) : "l"(b));
+    a0 = __fadd_rn(a0, b0), a1 = __fadd_rn(a1, b1);
+    asm("mov.b64 %0, {%1, %2};" : "=l"(a) : "f"(a0), "f"(a1));
+  }
 
   static __device__ __forceinline__ void zero(Acc& acc) {
     if constexpr (PAIRS) {
@@ -559,6 +572,8 @@ struct GemmKernel {
   using StageA = Stager<T, BM, BK, NT, SRC_A, Micro::LA, VEC, Micro::PA>;
   using StageB = Stager<T, BN, BK, NT, SRC_B, Micro::LB, VEC, Micro::PB>;
   static constexpr size_t SMEM_BYTES = (size_t)STAGES * (Micro::A_STAGE + Micro::B_STAGE) * sizeof(T);
+  // k split over a cluster: the micro-kernel supports it and the ring can hold a CTA's accumulators
+  static constexpr bool KSPLIT_OK = Micro::HAS_KSPLIT && SMEM_BYTES >= (size_t)BM * BN * sizeof(T);
 
   static __device__ __forceinline__ void run(const GemmArgs<T>& p) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -581,9 +596,21 @@ struct GemmKernel {
     const int64_t stepA = TA ? (int64_t)BK : (int64_t)BK * p.lda;  // advance by BK along k
     const int64_t stepB = TB ? (int64_t)BK * p.ldb : (int64_t)BK;
 
-    const int KT = (int)((p.k + BK - 1) / BK);
-    const int k_tail = (int)(p.k - (int64_t)(KT - 1) * BK);  // valid k-entries of the last slab
+    const int KT_all = (int)((p.k + BK - 1) / BK);
     const bool a_inside = (m_valid == BM), b_inside = (n_valid == BN);
+    // k split over a cluster: this CTA takes slabs [kt0, kt1) of the tile (possibly none)
+    int kt0 = 0, kt1 = KT_all;
+    if constexpr (KSPLIT_OK) {
+      if (p.ksplit > 1) {
+        const int per = (KT_all + p.ksplit - 1) / p.ksplit;
+        kt0 = min(KT_all, (int)blockIdx.z * per), kt1 = min(KT_all, kt0 + per);
+        gA += (int64_t)kt0 * stepA;
+        gB += (int64_t)kt0 * stepB;
+      }
+    }
+    const int KT = kt1 - kt0;
+    // valid k-entries of this CTA's last slab
+    const int k_tail = (kt1 == KT_all) ? (int)(p.k - (int64_t)(KT_all - 1) * BK) : BK;
 
     StageA stA;
     StageB stB;
@@ -592,7 +619,7 @@ struct GemmKernel {
 
     // beta != 0: pull this tile's old C values towards L2 now, so that the epilogue's loads overlap the k-loop
     // instead of paying the DRAM latency after it (this matters when k is only a few slabs).
-    if (p.beta != T(0)) {
+    if (p.beta != T(0) && (!KSPLIT_OK || blockIdx.z == 0)) {
       constexpr int LINE = 128 / (int)sizeof(T);   // elements per 128-byte line
       constexpr int LPC = (BM + LINE - 1) / LINE;  // lines per tile column
       for (int c = tid; c < BN * LPC; c += NT) {
@@ -697,6 +724,31 @@ struct GemmKernel {
       fill = (fill + 1 == STAGES) ? 0 : fill + 1;
     }
     cp_async_wait<0>();
+
+    // k split: the partial sums of ranks 1 .. ksplit-1 go through their (now idle) rings; rank 0 adds them in rank
+    // order, element by element, so the result does not depend on timing.  Every thread of every CTA of the
+    // cluster passes both cluster barriers: a split launch has no early exit (tri == 0).
+    if constexpr (KSPLIT_OK) {
+      if (p.ksplit > 1) {
+        unsigned long long* sAcc = reinterpret_cast<unsigned long long*>(smem_raw);
+        __syncthreads();  // every warp has finished reading the ring
+        if (blockIdx.z != 0) {
+#pragma unroll
+          for (int w = 0; w < Micro::ACC_WORDS; ++w) sAcc[w * NT + tid] = Micro::word(acc, w);
+        }
+        cluster_sync_all();  // partial sums are visible across the cluster
+        if (blockIdx.z == 0) {
+          for (int r = 1; r < p.ksplit; ++r) {
+            const uint32_t remote = cluster_map_shared(smem_u32(sAcc), (uint32_t)r);
+#pragma unroll
+            for (int w = 0; w < Micro::ACC_WORDS; ++w)
+              Micro::add_pair(Micro::word(acc, w), ld_cluster_b64(remote + (uint32_t)((w * NT + tid) * 8)));
+          }
+        }
+        cluster_sync_all();  // rank 0 has read everything: the other CTAs may leave
+        if (blockIdx.z != 0) return;
+      }
+    }
 
     // drain: fused alpha/beta epilogue
     T* Cb = p.C + (int64_t)blockIdx.y * p.batch_c;

@@ -15,6 +15,7 @@ struct VariantInfo {
   int tm = 8, tn = 8;  // FMA micro-kernels: accumulator block per thread
   double per_tile_extra_clks = 0.0;  // ramp-up and epilogue time of a tile that its co-resident CTAs do not cover
   double transpose_b_cost = 7.0;     // FMA micro-kernels: loss to the transposing copy of a k-contiguous B is cost/BM
+  bool can_ksplit = false;           // the kernel can split the k-loop of a tile over a thread-block cluster
 };
 
 template <typename T>
@@ -35,6 +36,20 @@ int launch_one(const GemmArgs<typename Kernel::T>& args, cudaStream_t stream) {
   const long long tiles = (long long)args.tiles_m * args.tiles_n;
   if (tiles <= 0 || tiles > 0x7fffffffLL) return B2_ERR_LAUNCH;
   const int batch = args.batch > 0 ? args.batch : 1;
+  if (args.ksplit > 1) {
+    // k split: grid.z = cluster size; the CTAs (tile, problem, 0 .. ksplit-1) form one cluster
+    if (!Kernel::KSPLIT_OK || args.ksplit > 8 || args.tri != 0) return B2_ERR_VARIANT;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)tiles, (unsigned)batch, (unsigned)args.ksplit);
+    cfg.blockDim = dim3(Kernel::NT, 1, 1);
+    cfg.dynamicSmemBytes = Kernel::SMEM_BYTES;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 1, attr[0].val.clusterDim.y = 1, attr[0].val.clusterDim.z = (unsigned)args.ksplit;
+    cfg.attrs = attr, cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kfn, args) == cudaSuccess ? B2_OK : B2_ERR_LAUNCH;
+  }
   kfn<<<dim3((unsigned)tiles, (unsigned)batch, 1), Kernel::NT, Kernel::SMEM_BYTES, stream>>>(args);
   return cudaGetLastError() == cudaSuccess ? B2_OK : B2_ERR_LAUNCH;
 }

@@ -257,6 +257,29 @@ def test_deterministic_bitwise(b2, kind):
     assert torch.equal(outs[0].view(torch.uint8), outs[1].view(torch.uint8))
 
 
+def test_sgemm_k_split_over_cluster(b2, oracle):
+    """fp32 problems of about a wave of 128 x 64 tiles are launched with the k-loop of every tile split over a
+    cluster of two CTAs (the second half reaches the first through distributed shared memory and is added in a
+    fixed order): ragged sizes, all transposes, padded and aligned leading dimensions, exact on integer data,
+    within the bound otherwise, the same bits on every run."""
+    import json
+    m, n, k = 1000, 1100, 777
+    cfg = json.loads(b2.b2_gemm_query_config(1, "N", "N", m, n, k, m, k, m))
+    if cfg["k_split"] < 2:
+        pytest.skip("the selector does not split this problem on this device")
+    for ta, tb in TRANS:
+        run_and_check(b2, oracle, "s", ta, tb, m, n, k, 0.7, -0.3, seed=51, pad=True)
+        run_and_check(b2, oracle, "s", ta, tb, m, n, k, 1.5, 0.5, dist="int9", seed=52, expect_exact=True)
+    run_and_check(b2, oracle, "s", "N", "N", m, n, 129, 1.0, 0.0, seed=53)   # 9 slabs: too few to split, same entry
+    A, lda, B, ldb, C, ldc = synth.gemm_inputs("N", "T", m, n, k, "uniform", 54, torch.float32)
+    outs = []
+    for _ in range(3):
+        Cd = C.cuda()
+        b2.b2_sgemm("N", "T", m, n, k, 0.7, A.cuda(), lda, B.cuda(), ldb, -0.3, Cd, ldc)
+        outs.append(Cd.cpu())
+    assert all(torch.equal(outs[0].view(torch.uint8), o.view(torch.uint8)) for o in outs[1:])
+
+
 # ---- complex 4M ------------------------------------------------------------------------------------
 
 def test_zgemm4m_small_full_all_transposes(b2, oracle):
