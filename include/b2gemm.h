@@ -106,8 +106,9 @@ const char* b2_variant_name(int dtype, int variant);
 
 /*
  * Writes a NUL-terminated JSON object describing what the selector would launch for this
- * problem (variant, CTA tile, kc, stages, micro-kernel, grid, shared memory) into json_out
- * (HOST memory, capacity cap bytes).  Returns 0, a negative argument index as above (dtype is
+ * problem (variant, CTA tile, kc, stages, micro-kernel, grid, and "k_split": over how many CTAs of a
+ * thread-block cluster the k-loop of each tile is divided, 1 = not divided; "grid" counts all CTAs) into
+ * json_out (HOST memory, capacity cap bytes).  Returns 0, a negative argument index as above (dtype is
  * argument 1 here, the rest shift by one), or B2_ERR_WORKSPACE when cap is too small.
  * Nothing is launched.  The tile derivation follows the paper's register-limit formula
  * (Section 5, "Limits imposed by registers") and pipeline-throughput estimate (Section 4).
