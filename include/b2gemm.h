@@ -12,8 +12,17 @@
  * with column-major storage, X(r, c) = X[r + c * ldx].
  *
  * Conventions shared by every entry point unless its comment says otherwise
- *   - A, B, C (and any workspace) are DEVICE pointers owned by the caller.  The library
- *     allocates nothing, keeps no state between calls and never frees anything.
+ *   - A, B, C (and any workspace) are DEVICE pointers owned by the caller.  No call allocates
+ *     or frees device or host memory.  What the library does hold, from the moment it is loaded
+ *     (or from the first call that needs it) until the process exits, is: the scratch array of
+ *     b2_zgemm4m_static (B2_ZGEMM4M_STATIC_BYTES of device memory on every GPU that loads the
+ *     library), two device status words (b2_device_status), per-device caches of symbol
+ *     addresses, shared-memory attributes and the SM count, and, for the host-buffer forms, two
+ *     helper streams and a few events per device.  None of it carries results from one call to
+ *     the next.
+ *   - Threads: the per-device caches are filled on first use through atomic slots and one-time
+ *     initialisers, so host threads may make their first calls concurrently.  Calls that share
+ *     an output or a workspace must be ordered by the caller.
  *   - Scalars are passed by value from the host.
  *   - Work is enqueued on `cuda_stream` (a cudaStream_t cast to void*; NULL = the legacy
  *     default stream) and the call returns without synchronising.
@@ -161,10 +170,14 @@ int b2_zgemm3m(char transa, char transb, int64_t m, int64_t n, int64_t k, const 
  *
  *   - Limit: b2_zgemm4m_workspace_bytes(transa, transb, m, n, k) must not exceed
  *     B2_ZGEMM4M_STATIC_BYTES (6 MiB: e.g. m = n = k = 256 needs 3 MiB, 360^3 just fits).
- *     Larger problems return B2_ERR_STATIC_LIMIT and launch nothing.
+ *     Larger problems return B2_ERR_STATIC_LIMIT and launch nothing.  The limit applies after
+ *     the argument checks and the quick returns, i.e. only to calls that really split planes:
+ *     an illegal argument still returns -i, and m == 0, n == 0, alpha == 0 or k == 0 behave as
+ *     in b2_zgemm4m whatever the sizes.
  *   - The call allocates and frees nothing, neither directly nor through a library.
  *   - The first call on each device looks up the array's device address (the device must be
- *     current); make that first call outside any stream capture.
+ *     current); make that first call outside any stream capture.  Host threads that make it
+ *     together each look the address up and store the same value.
  *   - All calls on a device share the one array, and it keeps the previous call's contents.
  *     Nothing in it has to start at zero (every plane element is written before it is read
  *     within a call), but two calls that overlap on the GPU -- different streams, or
@@ -213,8 +226,9 @@ int b2_sgemm_strided_batched(char transa, char transb, int64_t m, int64_t n, int
  *     b2_dtrsm:  solve op(A)*X = alpha*B (side 'L') or X*op(A) = alpha*B (side 'R');  X overwrites B
  * B is m x n, column-major, DEVICE memory, updated in place; A is DEVICE memory and is not modified.  alpha == 0
  * sets B to zero without reading A.  No singularity test is made (a zero on the diagonal divides by zero).
- * Method: recursive halving of the triangle puts all but the diagonal blocks of order <= 32 into calls of the
- * GEMM kernel; a diagonal block is handled by a substitution / product kernel with one warp per right-hand side.
+ * Method: recursive halving of the triangle puts all but the diagonal blocks of order <= 128 into calls of the
+ * GEMM kernel; a diagonal block is handled by a substitution / product kernel in which a warp holds four
+ * right-hand sides and walks the block's 32 x 32 sub-blocks in dependency order.
  * The order of summation therefore differs from column-by-column substitution; results satisfy the componentwise
  * residual bound of substitution, |op(A)*X - alpha*B| <= c*na*u*(|op(A)||X| + |alpha*B|), and are exact whenever
  * all intermediate values are exactly representable.
@@ -239,7 +253,8 @@ int b2_strsm(char side, char uplo, char transa, char diag, int64_t m, int64_t n,
  * fixed summation order (the paper, Section 2.1, fixes no order), so the b2_dgemm error bound applies and
  * integer-valued problems are bit-exact.
  *   splits     0 = chosen by the library (b2_gemm_splitk_auto: as many chunks as it takes to fill the SMs with
- *              64 x 64 tiles, each chunk at least 256 deep, at most 64); 1 = plain b2_dgemm; > k is cut to k.
+ *              64 x 64 tiles, each chunk at least 256 deep, at most 64); 1 = plain b2_dgemm; > k is cut to k,
+ *              > 65535 to 65535.
  *   workspace  DEVICE memory, 256-byte aligned, at least b2_gemm_splitk_workspace_bytes(dtype, m, n, k, splits)
  *              bytes (dtype 0 = fp64, 1 = fp32; 0 bytes when the call degenerates to the plain GEMM);
  *              owned by the caller, overwritten.
@@ -266,7 +281,8 @@ int b2_sgemm_splitk(char transa, char transb, int64_t m, int64_t n, int64_t k, f
  * Same arguments, quick returns and error codes as b2_sgemm, plus a DEVICE workspace of at least
  * b2_sgemm_tf32_workspace_bytes(terms, m, n, k) bytes (terms = 1 or 3), 256-byte aligned, owned by the caller
  * and overwritten (it receives the packed, rounded K-major panels of op(A) and op(B)); argument 14.
- * Any alignment and leading dimension of A, B, C is accepted.  Bounded device-side waits: b2_device_status.
+ * Any alignment and leading dimension of A, B, C is accepted; m and n up to 65535*64 and 3*k below 2^31
+ * (beyond that B2_ERR_VARIANT, nothing launched).  Bounded device-side waits: b2_device_status.
  */
 size_t b2_sgemm_tf32_workspace_bytes(int terms, int64_t m, int64_t n, int64_t k);
 int b2_sgemm_tf32x1(char transa, char transb, int64_t m, int64_t n, int64_t k, float alpha, const float* A,

@@ -90,7 +90,75 @@ def ptxas_report() -> str:
     return "\n".join(p.read_text() for p in sorted(BUILD_DIR.glob("*.ptxas.log")))
 
 
+def ptxas_summary() -> str:
+    """Markdown table of every kernel of the last build: registers, static shared memory, stack and spill bytes.
+
+    Parsed from the ``-Xptxas -v`` logs of the build; kernels that differ only in their transposition or
+    alignment template flags and use the same resources share a row.  The paper's spilling experiment
+    (Section 6.3) makes "no spills" a hard rule for the micro-kernel; the last column shows it holds.
+    """
+    import re
+    rows = {}
+    for log in sorted(BUILD_DIR.glob("*.ptxas.log")):
+        name = None
+        spill = stack = None
+        for line in log.read_text().splitlines():
+            m = re.search(r"Compiling entry function '([^']+)'", line)
+            if m:
+                name = m.group(1)
+                continue
+            m = re.search(r"(\d+) bytes stack frame, (\d+) bytes spill stores, (\d+) bytes spill loads", line)
+            if m and name:
+                stack, spill = int(m.group(1)), int(m.group(2)) + int(m.group(3))
+                continue
+            m = re.search(r"Used (\d+) registers(?:, used \d+ barriers)?(?:, (\d+) bytes smem)?", line)
+            if m and name:
+                regs, smem = int(m.group(1)), int(m.group(2) or 0)
+                pretty = _demangle(name)
+                key = (log.stem.replace(".ptxas", ""), _fold_flags(pretty), regs, smem, stack or 0, spill or 0)
+                rows[key] = rows.get(key, 0) + 1
+                name = None
+    out = ["| source file | kernel (template flags folded: `*` = any of true/false) | instances | registers | "
+           "static smem B | stack B | spill B |", "|---|---|---|---|---|---|---|"]
+    for (src, kern, regs, smem, stack, spill), count in sorted(rows.items()):
+        out.append(f"| {src}.cu | `{kern}` | {count} | {regs} | {smem} | {stack} | {spill} |")
+    total = sum(rows.values())
+    spilled = sum(c for k, c in rows.items() if k[5] or k[4])
+    out.append("")
+    out.append(f"{total} kernels, {spilled} with a stack frame or spills.")
+    return "\n".join(out)
+
+
+def _demangle(name: str) -> str:
+    exe = shutil.which("cu++filt") or shutil.which("c++filt")
+    if not exe:
+        return name
+    res = subprocess.run([exe, name], capture_output=True, text=True)
+    text = res.stdout.strip() or name
+    import re
+    text = re.sub(r"\(anonymous namespace\)::|<unnamed>::", "", text)
+    text = re.sub(r"^void ", "", text)
+    text = re.sub(r"\((?:int|bool|unsigned int|b2::Layout)\)", "", text)  # casts inside template argument lists
+    depth = 0
+    for i in range(len(text) - 1, -1, -1):  # drop the parameter list: the last top-level parenthesis group
+        if text[i] == ")":
+            depth += 1
+        elif text[i] == "(":
+            depth -= 1
+            if depth == 0:
+                text = text[:i]
+                break
+    return text.replace("b2::", "")
+
+
+def _fold_flags(pretty: str) -> str:
+    import re
+    return re.sub(r"\b(true|false)\b", "*", pretty)  # cu++filt prints bool template arguments as true/false
+
+
 if __name__ == "__main__":
     build(verbose=True, force="--force" in sys.argv)
     if "--ptxas" in sys.argv:
         print(ptxas_report())
+    if "--ptxas-summary" in sys.argv:
+        print(ptxas_summary())

@@ -1,5 +1,7 @@
 // C-ABI entry points of the real GEMM: argument checking, quick returns, variant selection.
 #include <cuda_runtime.h>
+
+#include <atomic>
 #include <math.h>
 #include <stdio.h>
 #include <string.h>
@@ -83,16 +85,16 @@ int check_gemm_args(char transa, char transb, int64_t m, int64_t n, int64_t k, c
   return 0;
 }
 
-static int sm_count_cached() {
-  static int cached[64] = {};
+int sm_count_cached() {
+  static std::atomic<int> cached[64];
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
-  if (cached[dev] == 0) {
-    int sms = 0;
+  int sms = cached[dev].load(std::memory_order_relaxed);
+  if (sms == 0) {
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) sms = 148;
-    cached[dev] = sms;
+    cached[dev].store(sms, std::memory_order_relaxed);
   }
-  return cached[dev];
+  return sms;
 }
 
 template <typename T>

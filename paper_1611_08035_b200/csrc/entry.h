@@ -26,6 +26,9 @@ int gemm_launch_checked(int variant, bool ta, bool tb, int64_t m, int64_t n, int
 int check_gemm_args(char transa, char transb, int64_t m, int64_t n, int64_t k, const void* A, int64_t lda,
                     const void* B, int64_t ldb, const void* C, int64_t ldc, bool reads_ab);
 
+// Multiprocessor count of the current device (queried once per device; 148 when the query fails).
+int sm_count_cached();
+
 inline size_t round_up(size_t x, size_t to) { return (x + to - 1) / to * to; }
 
 }  // namespace b2

@@ -17,17 +17,16 @@ using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, voi
                               const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                               CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
+EncodeFn lookup_encode_fn() {
+  void* p = nullptr;
+  cudaDriverEntryPointQueryResult q;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+      q == cudaDriverEntryPointSuccess)
+    return reinterpret_cast<EncodeFn>(p);
+  return nullptr;
+}
 EncodeFn encode_fn() {
-  static EncodeFn fn = nullptr;
-  static bool tried = false;
-  if (!tried) {
-    tried = true;
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
-        q == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<EncodeFn>(p);
-  }
+  static const EncodeFn fn = lookup_encode_fn();  // initialised once, thread-safe
   return fn;
 }
 
@@ -46,28 +45,30 @@ bool make_map(CUtensorMap* map, const double* base, int64_t rows, int64_t cols, 
 }
 
 int* status_pointer() {
-  static int* by_device[64] = {};
+  static std::atomic<int*> by_device[64];  // concurrent first calls store the same address
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
-  if (!by_device[dev]) {
+  int* cached = by_device[dev].load(std::memory_order_acquire);
+  if (!cached) {
     void* p = nullptr;
     if (cudaGetSymbolAddress(&p, g_device_status) != cudaSuccess) return nullptr;
-    by_device[dev] = static_cast<int*>(p);
+    cached = static_cast<int*>(p);
+    by_device[dev].store(cached, std::memory_order_release);
   }
-  return by_device[dev];
+  return cached;
 }
 
 template <class Kernel, int MIN_CTAS, bool TA, bool TB>
 int launch_tma_one(const GemmArgs<double>& a, cudaStream_t stream) {
-  static bool configured[64] = {};
+  static std::atomic<bool> configured[64];
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return B2_ERR_LAUNCH;
   auto kfn = gemm_tma_kernel<Kernel, MIN_CTAS>;
-  if (dev < 0 || dev >= 64 || !configured[dev]) {
+  if (dev < 0 || dev >= 64 || !configured[dev].load(std::memory_order_acquire)) {
     if (cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Kernel::SMEM_BYTES) !=
         cudaSuccess)
       return B2_ERR_LAUNCH;
-    if (dev >= 0 && dev < 64) configured[dev] = true;
+    if (dev >= 0 && dev < 64) configured[dev].store(true, std::memory_order_release);
   }
   int* status = status_pointer();
   if (!status) return B2_ERR_LAUNCH;
@@ -107,7 +108,8 @@ __global__ void wait_timeout_selftest_kernel(int* status) {
     mbar_fence_init();
   }
   __syncthreads();
-  if (threadIdx.x == 0 && !mbar_wait_bounded(&bar, 0, 1u << 12)) atomicExch(status, (int)B2_ERR_TIMEOUT);
+  // one millisecond, then give up
+  if (threadIdx.x == 0 && !mbar_wait_bounded(&bar, 0, 1000ull * 1000)) atomicExch(status, (int)B2_ERR_TIMEOUT);
 }
 
 template <bool TA, bool TB>

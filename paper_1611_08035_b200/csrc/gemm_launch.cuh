@@ -1,6 +1,8 @@
 // Host-side launch of one kernel variant: picks the (transA, transB, aligned) instantiation,
 // raises the dynamic shared-memory limit once per device and launches on the caller's stream.
 #pragma once
+#include <atomic>
+
 #include "b2gemm.h"
 #include "gemm_kernel.cuh"
 
@@ -23,15 +25,16 @@ using LaunchFn = int (*)(const GemmArgs<T>& args, bool ta, bool tb, bool aligned
 
 template <class Kernel, int MIN_CTAS>
 int launch_one(const GemmArgs<typename Kernel::T>& args, cudaStream_t stream) {
-  static bool configured[64] = {};
+  // one flag per device; threads that get here together both set the (idempotent) attribute
+  static std::atomic<bool> configured[64];
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return B2_ERR_LAUNCH;
   auto kfn = gemm_kernel<Kernel, MIN_CTAS>;
-  if (dev < 0 || dev >= 64 || !configured[dev]) {
+  if (dev < 0 || dev >= 64 || !configured[dev].load(std::memory_order_acquire)) {
     if (cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Kernel::SMEM_BYTES) !=
         cudaSuccess)
       return B2_ERR_LAUNCH;
-    if (dev >= 0 && dev < 64) configured[dev] = true;
+    if (dev >= 0 && dev < 64) configured[dev].store(true, std::memory_order_release);
   }
   const long long tiles = (long long)args.tiles_m * args.tiles_n;
   if (tiles <= 0 || tiles > 0x7fffffffLL) return B2_ERR_LAUNCH;

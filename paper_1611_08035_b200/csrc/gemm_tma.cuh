@@ -44,11 +44,27 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
       : "memory");
   return done != 0;
 }
-// Bounded wait: false when the phase did not complete within kSpinLimit polls.
-constexpr uint32_t kSpinLimit = 1u << 24;
-__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, uint32_t limit = kSpinLimit) {
-  for (uint32_t spin = 0; spin < limit; ++spin)
-    if (mbar_try_wait(bar, parity)) return true;
+// Bounded wait: false when the phase did not complete within limit_ns nanoseconds of wall time.  The bound is a
+// time (the global nanosecond timer), not a number of polls, because one try_wait may itself block for an
+// implementation-defined interval.  A wait that succeeds at once never reads the timer; after that the timer is
+// read once per 32 polls.  kWaitLimitNs is far beyond any legitimate wait of these kernels (a slab arrives within
+// microseconds) and still bounds a stuck CTA to about a second; kDrainLimitNs bounds the waits for copies that are
+// already in flight when a kernel gives up.
+constexpr uint64_t kWaitLimitNs = 1000ull * 1000 * 1000;
+constexpr uint64_t kDrainLimitNs = 50ull * 1000 * 1000;
+__device__ __forceinline__ uint64_t global_timer_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, uint64_t limit_ns = kWaitLimitNs) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const uint64_t t0 = global_timer_ns();
+  do {
+#pragma unroll 1
+    for (int poll = 0; poll < 32; ++poll)
+      if (mbar_try_wait(bar, parity)) return true;
+  } while (global_timer_ns() - t0 < limit_ns);
   return false;
 }
 // One 2-D box from global (through the tensor map) to shared memory, completion counted on `bar`.
@@ -171,7 +187,7 @@ struct GemmTmaKernel {
       atomicExch(status, (int)B2_ERR_TIMEOUT);
       if (tid == 0) {
         for (int kt = waited; kt < issued; ++kt)
-          (void)mbar_wait_bounded(&full[kt % STAGES], (uint32_t)((kt / STAGES) & 1));
+          (void)mbar_wait_bounded(&full[kt % STAGES], (uint32_t)((kt / STAGES) & 1), kDrainLimitNs);
       }
       return;
     }

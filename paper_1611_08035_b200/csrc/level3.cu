@@ -40,7 +40,8 @@ __global__ void batch_scale_kernel(int64_t m, int64_t n, T beta, T* C, int64_t l
 
 unsigned blocks_for(int64_t total) {
   int64_t b = (total + 255) / 256;
-  if (b > 148 * 16) b = 148 * 16;
+  const int64_t cap = (int64_t)sm_count_cached() * 16;
+  if (b > cap) b = cap;
   return (unsigned)(b < 1 ? 1 : b);
 }
 
@@ -147,7 +148,7 @@ int64_t splitk_pitch(int64_t m) {
 int splitk_auto(int64_t m, int64_t n, int64_t k) {
   if (m <= 0 || n <= 0 || k <= 0) return 1;
   const int64_t tiles = ((m + 63) / 64) * ((n + 63) / 64);
-  const int64_t slots = 148 * 4;  // resident 64 x 64 tiles
+  const int64_t slots = (int64_t)sm_count_cached() * 4;  // resident 64 x 64 tiles
   int64_t s = slots / tiles;
   if (s > k / 256) s = k / 256;  // every chunk at least 256 deep
   if (s > 64) s = 64;
@@ -164,6 +165,7 @@ int gemm_splitk(char transa, char transb, int64_t m, int64_t n, int64_t k, T alp
   if (splits < 0) return -14;
   if (splits == 0) splits = splitk_auto(m, n, k);
   if (splits > k) splits = k > 0 ? (int)k : 1;
+  if (splits > 65535) splits = 65535;  // the chunks are the second grid dimension of one launch
   if (scale_only || splits <= 1 || m == 0 || n == 0)
     return gemm_entry<T>(B2_VARIANT_AUTO, transa, transb, m, n, k, alpha, A, lda, B, ldb, beta, C, ldc, cuda_stream);
   const int64_t chunk = ((k + splits - 1) / splits + kSplitChunkUnit - 1) / kSplitChunkUnit * kSplitChunkUnit;
@@ -197,6 +199,7 @@ size_t splitk_workspace_bytes(int64_t m, int64_t n, int64_t k, int splits) {
   if (m <= 0 || n <= 0 || k <= 0 || splits < 0) return 0;
   if (splits == 0) splits = splitk_auto(m, n, k);
   if (splits > k) splits = (int)k;
+  if (splits > 65535) splits = 65535;
   if (splits <= 1) return 0;
   return (size_t)splits * (size_t)splitk_pitch<T>(m) * (size_t)n * sizeof(T);
 }

@@ -19,6 +19,8 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 
+#include <atomic>
+
 #include "b2gemm.h"
 #include "entry.h"
 #include "gemm_tma.cuh"
@@ -222,6 +224,7 @@ __global__ void __launch_bounds__(128, MINB)
   const uint32_t tmem_d = *tmem_slot;
 
   bool ok = true;
+  bool committed = false;  // issuing thread: the accumulator's completion has been committed to `accum`
   if (warp == 0 && lane == 0) {
     // ---- producer: TMA boxes of 32 (k) x 128 rows of both panels
     int issued = 0;
@@ -241,7 +244,8 @@ __global__ void __launch_bounds__(128, MINB)
       // let the copies still in flight land: the latest fill of every slot
       for (int s = 0; s < TSTAGES; ++s) {
         const int last = ((issued - 1 - s) / TSTAGES) * TSTAGES + s;  // last slab that went to slot s
-        if (issued > s && last >= 0) (void)mbar_wait_bounded(&full[s], (uint32_t)((last / TSTAGES) & 1));
+        if (issued > s && last >= 0)
+          (void)mbar_wait_bounded(&full[s], (uint32_t)((last / TSTAGES) & 1), kDrainLimitNs);
       }
     }
   } else if (warp == 1 && lane == 0) {
@@ -265,6 +269,7 @@ __global__ void __launch_bounds__(128, MINB)
     }
     if (ok) {
       umma_commit(accum);  // the accumulator is complete once everything issued has finished
+      committed = true;
     } else {
       atomicExch(p.status, (int)B2_ERR_TIMEOUT);
     }
@@ -272,9 +277,13 @@ __global__ void __launch_bounds__(128, MINB)
   __syncwarp();
 
   // ---- epilogue: every warp reads its 32 accumulator rows, 16 columns at a time
+  bool done = true;
   if (KT > 0) {
-    // warp-uniform verdict: the accumulator load below is a warp-wide instruction
-    const bool done = __all_sync(0xffffffffu, mbar_wait_bounded(accum, 0) ? 1 : 0) != 0;
+    // Warp-uniform verdict: the accumulator load below is a warp-wide instruction.  Most threads start this wait
+    // at kernel entry, so its limit grows with the length of the k-loop it has to outlast (a slab of this tile
+    // takes well under a microsecond of tensor-pipe time; four are allowed).
+    const uint64_t accum_limit = kWaitLimitNs + (uint64_t)KT * 4096ull;
+    done = __all_sync(0xffffffffu, mbar_wait_bounded(accum, 0, accum_limit) ? 1 : 0) != 0;
     tc_fence_after();
     if (done) {
       const int64_t row = m0 + warp * 32 + lane;
@@ -312,7 +321,11 @@ __global__ void __launch_bounds__(128, MINB)
     }
   }
 
-  // ---- common exit: free the tensor memory
+  // ---- common exit: free the tensor memory.  The barrier below is reached by the producer only after its copies
+  // have landed (or their bounded waits ran out).  If the epilogue gave up although the issuing thread had
+  // committed the accumulator, multiply-adds may still be running: that thread waits for them once more (bounded)
+  // before the tensor memory they write is freed.
+  if (warp == 1 && lane == 0 && !done && committed) (void)mbar_wait_bounded(accum, 0, kWaitLimitNs);
   tc_fence_before();
   __syncthreads();
   if (warp == 1) tmem_dealloc(tmem_d, TBN);
@@ -321,17 +334,16 @@ __global__ void __launch_bounds__(128, MINB)
 using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                               const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                               CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeFn tf32_lookup_encode_fn() {
+  void* ptr = nullptr;
+  cudaDriverEntryPointQueryResult q;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) == cudaSuccess &&
+      q == cudaDriverEntryPointSuccess)
+    return reinterpret_cast<EncodeFn>(ptr);
+  return nullptr;
+}
 EncodeFn tf32_encode_fn() {
-  static EncodeFn fn = nullptr;
-  static bool tried = false;
-  if (!tried) {
-    tried = true;
-    void* ptr = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) == cudaSuccess &&
-        q == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<EncodeFn>(ptr);
-  }
+  static const EncodeFn fn = tf32_lookup_encode_fn();  // initialised once, thread-safe
   return fn;
 }
 
@@ -352,13 +364,13 @@ bool t_is_n(char c) { return c == 'N' || c == 'n'; }
 
 template <int TBN, int TSTAGES, int MINB = 1>
 int launch_tf32(const Tf32Args& a, const float* PA, const float* PB, int64_t pitch, int dev, cudaStream_t st) {
-  static bool configured[64] = {};
+  static std::atomic<bool> configured[64];
   auto kfn = sgemm_tf32_kernel<TBN, TSTAGES, MINB>;
   constexpr size_t smem = Tf32Cfg<TBN, TSTAGES>::SMEM_BYTES;
-  if (!configured[dev]) {
+  if (!configured[dev].load(std::memory_order_acquire)) {
     if (cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
       return B2_ERR_LAUNCH;
-    configured[dev] = true;
+    configured[dev].store(true, std::memory_order_release);
   }
   CUtensorMap mapA, mapB;
   if (!panel_map(&mapA, PA, a.m, pitch, TBM) || !panel_map(&mapB, PB, a.n, pitch, TBN)) return B2_ERR_LAUNCH;
@@ -391,20 +403,23 @@ int sgemm_tf32(int terms, char transa, char transb, int64_t m, int64_t n, int64_
   if (m == 0 || n == 0) return B2_OK;
   if (scale_only)  // C := beta*C needs no tensor cores
     return gemm_entry<float>(B2_VARIANT_AUTO, transa, transb, m, n, k, alpha, A, lda, B, ldb, beta, C, ldc, cuda_stream);
-  if (m > 0x7fffffffLL || n > 0x7fffffffLL || k > 0x2aaaaaaaLL) return B2_ERR_VARIANT;
+  // 32-bit tile coordinates; the pack kernel walks the rows of an operand in 64-row blocks of the grid's second
+  // dimension (at most 65535 blocks)
+  constexpr int64_t kMaxRows = 65535LL * 64;
+  if (m > kMaxRows || n > kMaxRows || k > 0x2aaaaaaaLL) return B2_ERR_VARIANT;
   const PackPlan pl = pack_plan(terms, m, n, k);
   if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255) != 0 || ws_bytes < pl.total) return B2_ERR_WORKSPACE;
   cudaStream_t st = (cudaStream_t)cuda_stream;
   float* PA = reinterpret_cast<float*>(ws);
   float* PB = reinterpret_cast<float*>(static_cast<char*>(ws) + pl.off_b);
 
-  static int* status_by_device[64] = {};
+  static std::atomic<int*> status_by_device[64];
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return B2_ERR_LAUNCH;
-  if (!status_by_device[dev]) {
+  if (!status_by_device[dev].load(std::memory_order_acquire)) {
     void* sp = nullptr;
     if (cudaGetSymbolAddress(&sp, g_tf32_status) != cudaSuccess) return B2_ERR_LAUNCH;
-    status_by_device[dev] = static_cast<int*>(sp);
+    status_by_device[dev].store(static_cast<int*>(sp), std::memory_order_release);
   }
 
   // step 1: pack.  op(A)(i, p): A[i + p*lda] (N) or A[p + i*lda] (T);  op(B)^T(j, p): B[p + j*ldb] (N) or B[j + p*ldb] (T)
@@ -432,13 +447,7 @@ int sgemm_tf32(int terms, char transa, char transb, int64_t m, int64_t n, int64_
     // with a 2-stage ring (96 KB) and 256 of the 512 tensor-memory columns, so that one CTA's epilogue and ramp-up
     // run under the other's multiply-adds.  Measured (TFLOP/s, packing included, against one CTA with 4 stages):
     // 3072^3 440 / 386, 4096^3 476 / 412, 8192^3 663 / 592, three-term 4096^3 200 / 187, 8192^3 225 / 228.
-    static int sms_by_device[64] = {};
-    if (sms_by_device[dev] == 0) {
-      int sms = 0;
-      if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) sms = 148;
-      sms_by_device[dev] = sms;
-    }
-    if (wide_tiles > sms_by_device[dev] && a.kt <= 512) return launch_tf32<256, 2, 2>(a, PA, PB, pl.pitch, dev, st);
+    if (wide_tiles > sm_count_cached() && a.kt <= 512) return launch_tf32<256, 2, 2>(a, PA, PB, pl.pitch, dev, st);
     return launch_tf32<256, 4>(a, PA, PB, pl.pitch, dev, st);
   }
   return launch_tf32<128, 6>(a, PA, PB, pl.pitch, dev, st);

@@ -6,6 +6,8 @@
 //     Cr = A'r*Br - A'i*Bi + (beta*C)r,      Ci = A'r*Bi + A'i*Br + (beta*C)i.
 // Steps: split kernels write the six planes into the caller's workspace, four real GEMMs
 // accumulate into the two C planes, a merge kernel interleaves them back into C.
+#include <atomic>
+
 #include "b2gemm.h"
 #include "entry.h"
 
@@ -130,10 +132,19 @@ extern "C" size_t b2_zgemm4m_workspace_bytes(char transa, char transb, int64_t m
   return make_plan(transa, transb, m, n, k).total;
 }
 
-extern "C" int b2_zgemm4m(char transa, char transb, int64_t m, int64_t n, int64_t k, const double alpha[2],
-                          const void* A, int64_t lda, const void* B, int64_t ldb, const double beta[2], void* C,
-                          int64_t ldc, void* workspace, size_t workspace_bytes, void* cuda_stream) {
-  using namespace b2;
+namespace b2 {
+namespace {
+// Where the six planes of a 4M call live: the caller's workspace, or the array built into the library.
+struct Scratch {
+  void* workspace;
+  size_t workspace_bytes;
+  bool built_in;  // resolve the built-in array (after the argument checks and quick returns) instead
+};
+void* builtin_scratch();  // device address of the built-in array on the current device (nullptr on failure)
+
+int zgemm4m_run(char transa, char transb, int64_t m, int64_t n, int64_t k, const double alpha[2], const void* A,
+                int64_t lda, const void* B, int64_t ldb, const double beta[2], void* C, int64_t ldc, Scratch scratch,
+                void* cuda_stream) {
   if (!is_op(transa)) return -1;
   if (!is_op(transb)) return -2;
   if (!alpha) return -6;
@@ -152,8 +163,15 @@ extern "C" int b2_zgemm4m(char transa, char transb, int64_t m, int64_t n, int64_
     return cudaGetLastError() == cudaSuccess ? B2_OK : B2_ERR_LAUNCH;
   }
   const Plan p = make_plan(transa, transb, m, n, k);
-  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) != 0 || workspace_bytes < p.total)
+  void* workspace = scratch.workspace;
+  if (scratch.built_in) {
+    // only a call that really splits planes is held to the size of the built-in array
+    if (p.total > (size_t)B2_ZGEMM4M_STATIC_BYTES) return B2_ERR_STATIC_LIMIT;
+    workspace = builtin_scratch();
+    if (!workspace) return B2_ERR_LAUNCH;
+  } else if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) != 0 || scratch.workspace_bytes < p.total) {
     return B2_ERR_WORKSPACE;
+  }
   char* w = static_cast<char*>(workspace);
   double* Apr = reinterpret_cast<double*>(w + p.off[0]);
   double* Api = reinterpret_cast<double*>(w + p.off[1]);
@@ -186,6 +204,15 @@ extern "C" int b2_zgemm4m(char transa, char transb, int64_t m, int64_t n, int64_
   if (rc) return rc;
   zmerge_kernel<<<grid_for(m, n), 256, 0, st>>>(m, n, Cr, Ci, p.lpc, Cz, ldc);
   return cudaGetLastError() == cudaSuccess ? B2_OK : B2_ERR_LAUNCH;
+}
+}  // namespace
+}  // namespace b2
+
+extern "C" int b2_zgemm4m(char transa, char transb, int64_t m, int64_t n, int64_t k, const double alpha[2],
+                          const void* A, int64_t lda, const void* B, int64_t ldb, const double beta[2], void* C,
+                          int64_t ldc, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  return b2::zgemm4m_run(transa, transb, m, n, k, alpha, A, lda, B, ldb, beta, C, ldc,
+                         b2::Scratch{workspace, workspace_bytes, false}, cuda_stream);
 }
 
 // ---- 3M: three real products instead of four ----------------------------------------------------
@@ -249,24 +276,30 @@ extern "C" int b2_zgemm3m(char transa, char transb, int64_t m, int64_t n, int64_
 // ---- b2_zgemm4m without a caller-provided workspace -------------------------------------------
 // The scratch planes live in the library image.  In host code the array's name is only a
 // host-side stand-in for the symbol, not a device address: the address each device maps it
-// to is looked up once per device with cudaGetSymbolAddress and cached.
+// to is looked up once per device (with that device current) by cudaGetSymbolAddress and cached.
+// Two host threads that make their first call on a device together both look the address up and
+// store the same value (atomic slots), which is harmless.
 static __device__ __align__(256) unsigned char g_zgemm4m_scratch[B2_ZGEMM4M_STATIC_BYTES];
+
+namespace b2 {
+namespace {
+void* builtin_scratch() {
+  static std::atomic<void*> by_device[64];
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  void* ptr = by_device[dev].load(std::memory_order_acquire);
+  if (!ptr) {
+    if (cudaGetSymbolAddress(&ptr, g_zgemm4m_scratch) != cudaSuccess || !ptr) return nullptr;
+    by_device[dev].store(ptr, std::memory_order_release);
+  }
+  return ptr;
+}
+}  // namespace
+}  // namespace b2
 
 extern "C" int b2_zgemm4m_static(char transa, char transb, int64_t m, int64_t n, int64_t k, const double alpha[2],
                                  const void* A, int64_t lda, const void* B, int64_t ldb, const double beta[2],
                                  void* C, int64_t ldc, void* cuda_stream) {
-  using namespace b2;
-  static void* scratch_by_device[64] = {};
-  if (is_op(transa) && is_op(transb) && m >= 0 && n >= 0 && k >= 0 &&
-      make_plan(transa, transb, m, n, k).total > (size_t)B2_ZGEMM4M_STATIC_BYTES)
-    return B2_ERR_STATIC_LIMIT;
-  int dev = -1;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return B2_ERR_LAUNCH;
-  if (!scratch_by_device[dev]) {
-    void* ptr = nullptr;
-    if (cudaGetSymbolAddress(&ptr, g_zgemm4m_scratch) != cudaSuccess || !ptr) return B2_ERR_LAUNCH;
-    scratch_by_device[dev] = ptr;
-  }
-  return b2_zgemm4m(transa, transb, m, n, k, alpha, A, lda, B, ldb, beta, C, ldc, scratch_by_device[dev],
-                    (size_t)B2_ZGEMM4M_STATIC_BYTES, cuda_stream);
+  return b2::zgemm4m_run(transa, transb, m, n, k, alpha, A, lda, B, ldb, beta, C, ldc,
+                         b2::Scratch{nullptr, 0, true}, cuda_stream);
 }

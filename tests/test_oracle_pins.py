@@ -391,6 +391,58 @@ def test_conjugate_transposes_of_the_complex_oracle(oracle):
     assert np.allclose(d.real, np.sum(np.abs(A2) ** 2, axis=0), rtol=1e-14)
 
 
+def test_complex_wide_oracle_magnitude_sum_and_result_exact(oracle):
+    """The wide complex oracle's two outputs against independent evaluations, for all nine op pairs (N/T/C).
+
+    S, the magnitude sum every complex tolerance is built from, against exact rational arithmetic:
+    S_ij = (|ar|+|ai|) sum_p (|Ar|+|Ai|)_ip (|Br|+|Bi|)_pj + (|br|+|bi|)(|Cr|+|Ci|)_ij, to 1e-12 relative; a scaled
+    sum, a dropped absolute value or a forgotten alpha/beta factor all move it by far more.  Chi, the rounded wide
+    result, against numpy on integer data (where the exact result is representable) bit for bit, and against the
+    rational result on general data within one rounding of S."""
+    rng = np.random.default_rng(31)
+    m, n, k = 4, 3, 9
+    F = lambda x: Fraction(float(x))
+    for ta in "NTC":
+        for tb in "NTC":
+            ra, ca = (m, k) if ta == "N" else (k, m)
+            rb, cb = (k, n) if tb == "N" else (n, k)
+            A2 = rng.uniform(-1, 1, (ra, ca)) + 1j * rng.uniform(-1, 1, (ra, ca))
+            B2 = rng.uniform(-1, 1, (rb, cb)) + 1j * rng.uniform(-1, 1, (rb, cb))
+            C2 = rng.uniform(-1, 1, (m, n)) + 1j * rng.uniform(-1, 1, (m, n))
+            alpha, beta = (0.75 - 0.5j), (-0.25 + 1.5j)
+            A, B, C = store(A2, ra + 2, np.nan), store(B2, rb + 1, np.nan), store(C2, m + 3, SENTINEL)
+            hi, S = oracle.ref_gemm_hi(ta, tb, m, n, k, alpha, A, ra + 2, B, rb + 1, beta, C, m + 3)
+            hi2, S2 = unstore(hi, m, n, m), unstore(S, m, n, m)
+            opA, opB = _zop(A2, ta), _zop(B2, tb)
+            for i in range(m):
+                for j in range(n):
+                    mag = sum((abs(F(opA[i, p].real)) + abs(F(opA[i, p].imag))) *
+                              (abs(F(opB[p, j].real)) + abs(F(opB[p, j].imag))) for p in range(k))
+                    s_exact = (abs(F(alpha.real)) + abs(F(alpha.imag))) * mag + \
+                        (abs(F(beta.real)) + abs(F(beta.imag))) * (abs(F(C2[i, j].real)) + abs(F(C2[i, j].imag)))
+                    assert abs(F(S2[i, j]) - s_exact) <= Fraction(1, 10 ** 12) * s_exact, (ta, tb, i, j)
+                    sr = sum(F(opA[i, p].real) * F(opB[p, j].real) - F(opA[i, p].imag) * F(opB[p, j].imag)
+                             for p in range(k))
+                    si = sum(F(opA[i, p].real) * F(opB[p, j].imag) + F(opA[i, p].imag) * F(opB[p, j].real)
+                             for p in range(k))
+                    wr = F(alpha.real) * sr - F(alpha.imag) * si + F(beta.real) * F(C2[i, j].real) - \
+                        F(beta.imag) * F(C2[i, j].imag)
+                    wi = F(alpha.real) * si + F(alpha.imag) * sr + F(beta.real) * F(C2[i, j].imag) + \
+                        F(beta.imag) * F(C2[i, j].real)
+                    tol = Fraction(2.0 ** -52) * s_exact  # long double accumulation, then one rounding to double
+                    assert abs(F(hi2[i, j].real) - wr) <= tol and abs(F(hi2[i, j].imag) - wi) <= tol, (ta, tb, i, j)
+            # integer data: the exact result is a double, so Chi must equal numpy's bit for bit
+            A2, B2, C2 = _zint(rng, (ra, ca)), _zint(rng, (rb, cb)), _zint(rng, (m, n))
+            alpha, beta = 2 - 1j, 0.5 + 0.5j
+            hi, S = oracle.ref_gemm_hi(ta, tb, m, n, k, alpha, store(A2, ra, np.nan), ra, store(B2, rb, np.nan), rb,
+                                       beta, store(C2, m, SENTINEL), m)
+            assert np.array_equal(unstore(hi, m, n, m), alpha * (_zop(A2, ta) @ _zop(B2, tb)) + beta * C2)
+            want_s = 3.0 * ((np.abs(_zop(A2, ta).real) + np.abs(_zop(A2, ta).imag)) @
+                            (np.abs(_zop(B2, tb).real) + np.abs(_zop(B2, tb).imag))) + \
+                1.0 * (np.abs(C2.real) + np.abs(C2.imag))
+            assert np.array_equal(unstore(S, m, n, m), want_s)  # small integers and halves: exact
+
+
 def test_3m_steps_against_the_definition(oracle):
     """3M against direct complex arithmetic on general data: both components within 2*(3k+6)*u*S of the wide
     result (S = sum (|Ar|+|Ai|)(|Br|+|Bi|) scaled by |alpha| plus the beta term), and the real component, which
