@@ -80,6 +80,11 @@ int b2_sgemm(char transa, char transb, int64_t m, int64_t n, int64_t k, float al
  * The same two operations with an explicit kernel variant, 0 <= variant < b2_variant_count(dtype),
  * or B2_VARIANT_AUTO.  Used by tests and benchmarks to exercise every micro-kernel; a variant
  * that cannot serve the given shape/alignment returns B2_ERR_VARIANT and launches nothing.
+ * An explicit variant is launched with one CTA per tile; variant + 256*s (s = 2 or 4) asks for
+ * the k-loop of every tile to be split over a thread-block cluster of s CTAs, whose partial
+ * sums are added in rank order through distributed shared memory (Section 2's kc loop, cut in
+ * s pieces; same error bound, bit-exact on integer-valued data, the same bits on every run).
+ * Variants that cannot split (the TMA-staged and scalar-FMA ones) return B2_ERR_VARIANT.
  */
 int b2_dgemm_variant(int variant, char transa, char transb, int64_t m, int64_t n, int64_t k, double alpha,
                      const double* A, int64_t lda, const double* B, int64_t ldb, double beta, double* C,

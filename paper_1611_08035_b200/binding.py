@@ -392,6 +392,14 @@ def b2_sgemm_tf32(terms, transa, transb, m, n, k, alpha, A, lda, B, ldb, beta, C
     return rc
 
 
+def b2_sgemm_tf32x1(transa, transb, m, n, k, alpha, A, lda, B, ldb, beta, C, ldc, workspace, check=True) -> int:
+    return b2_sgemm_tf32(1, transa, transb, m, n, k, alpha, A, lda, B, ldb, beta, C, ldc, workspace, check)
+
+
+def b2_sgemm_tf32x3(transa, transb, m, n, k, alpha, A, lda, B, ldb, beta, C, ldc, workspace, check=True) -> int:
+    return b2_sgemm_tf32(3, transa, transb, m, n, k, alpha, A, lda, B, ldb, beta, C, ldc, workspace, check)
+
+
 def b2_syrk(uplo, trans, n, k, alpha, A, lda, beta, C, ldc, check=True) -> int:
     """Symmetric rank-k update on the uplo triangle of C (b2_dsyrk / b2_ssyrk by dtype); device tensors."""
     if C is not None and C.dtype == torch.float32:

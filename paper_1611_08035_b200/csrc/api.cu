@@ -22,6 +22,7 @@ int launch_f64_v5(const GemmArgs<double>&, bool, bool, bool, cudaStream_t);
 int launch_f64_v6(const GemmArgs<double>&, bool, bool, bool, cudaStream_t);
 int launch_f64_t32(const GemmArgs<double>&, bool, bool, bool, cudaStream_t);
 int launch_f64_tma_t32(const GemmArgs<double>&, bool, bool, bool, cudaStream_t);
+int launch_f64_w8(const GemmArgs<double>&, bool, bool, bool, cudaStream_t);
 int launch_f32_v0(const GemmArgs<float>&, bool, bool, bool, cudaStream_t);
 int launch_f32_v1(const GemmArgs<float>&, bool, bool, bool, cudaStream_t);
 int launch_f32_v2(const GemmArgs<float>&, bool, bool, bool, cudaStream_t);
@@ -41,10 +42,11 @@ const VariantInfo kF64Info[] = {
     {"dmma_tma_128x128x16_s4", "dmma_tma", 128, 128, 16, 4, 256, 1, 0.95},
     {"dmma_32x32x16_s3", "dmma", 32, 32, 16, 3, 128, 6, 0.80},
     {"dmma_tma_32x32x16_s3", "dmma_tma", 32, 32, 16, 3, 128, 6, 0.80},
+    {"dmma_w8_64x64x16_s3", "dmma", 64, 64, 16, 3, 256, 3, 0.92},
 };
 const LaunchFn<double> kF64Launch[] = {launch_f64_v0, launch_f64_v1, launch_f64_v2, launch_f64_v3,
                                        launch_f64_v4, launch_f64_v5, launch_f64_v6, launch_f64_t32,
-                                       launch_f64_tma_t32};
+                                       launch_f64_tma_t32, launch_f64_w8};
 const VariantInfo kF32Info[] = {
     {"ffma2_t16x8_128x128x16_s3", "ffma2", 128, 128, 16, 3, 128, 2, 0.782, 16, 8, 3500.0, 11.0},
     {"ffma2_128x64x16_s4", "ffma2", 128, 64, 16, 4, 128, 3, 0.795, 8, 8, 0.0, 5.8, true},
@@ -200,7 +202,7 @@ int gemm_launch_checked(int variant, bool ta, bool tb, int64_t m, int64_t n, int
   constexpr int64_t kVec = 16 / (int64_t)sizeof(T);
   const bool aligned = operands_aligned(A, lda, B, ldb) &&
                        (ex.batch <= 1 || (ex.stride_a % kVec == 0 && ex.stride_b % kVec == 0));
-  int ksplit = 1;
+  int ksplit = ex.ksplit > 0 ? ex.ksplit : 1;
   if (variant == B2_VARIANT_AUTO)
     variant = choose_variant<T>(m, n, k, aligned, ex.batch, ta, tb, ex.tri == 0 ? &ksplit : nullptr);
   GemmArgs<T> args;
@@ -234,6 +236,13 @@ int gemm_entry(int variant, char transa, char transb, int64_t m, int64_t n, int6
   const bool scale_only = (alpha == T(0) || k == 0);
   const int bad = check_gemm_args(transa, transb, m, n, k, A, lda, B, ldb, C, ldc, !scale_only);
   if (bad) return bad;
+  // an explicit variant may carry a k split request: variant + 256 * (CTAs per tile)
+  GemmExtra ex;
+  if (variant >= 256) {
+    ex.ksplit = variant >> 8;
+    variant &= 255;
+    if (ex.ksplit != 2 && ex.ksplit != 4) return B2_ERR_VARIANT;
+  }
   if (variant != B2_VARIANT_AUTO && (variant < 0 || variant >= variant_count_t<T>())) return B2_ERR_VARIANT;
   if (m == 0 || n == 0) return B2_OK;
   cudaStream_t stream = (cudaStream_t)cuda_stream;
@@ -248,7 +257,7 @@ int gemm_entry(int variant, char transa, char transb, int64_t m, int64_t n, int6
     return cudaGetLastError() == cudaSuccess ? B2_OK : B2_ERR_LAUNCH;
   }
   return gemm_launch_checked<T>(variant, is_t(transa), is_t(transb), m, n, k, alpha, A, lda, B, ldb, beta, C, ldc,
-                                GemmExtra(), stream);
+                                ex, stream);
 }
 
 // Explicit instantiations used by the other translation units (complex and host-buffer entries).

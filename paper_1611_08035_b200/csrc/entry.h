@@ -15,6 +15,7 @@ struct GemmExtra {
   int tri = 0;
   int batch = 1;
   int64_t stride_a = 0, stride_b = 0, stride_c = 0;
+  int ksplit = 0;  // k split of every tile over a cluster: 0 = the selector's choice (automatic variant) or none
 };
 // Variant choice and launch of an already checked, non-trivial problem (m, n, k > 0, alpha != 0); ta/tb: transposed.
 template <typename T>

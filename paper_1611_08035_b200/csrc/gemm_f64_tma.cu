@@ -86,7 +86,7 @@ int launch_tma_one(const GemmArgs<double>& a, cudaStream_t stream) {
 template <template <bool, bool> class MicroT, int STAGES, int MIN_CTAS>
 int launch_tma(const GemmArgs<double>& args_in, bool ta, bool tb, bool aligned, cudaStream_t s) {
   // tensor maps need 16-byte aligned bases and row pitches; coordinates are 32-bit
-  if (!aligned || args_in.batch > 1) return B2_ERR_VARIANT;
+  if (!aligned || args_in.batch > 1 || args_in.ksplit > 1) return B2_ERR_VARIANT;
   if (args_in.m > 0x7fffffffLL || args_in.n > 0x7fffffffLL || args_in.k > 0x7fffffffLL) return B2_ERR_VARIANT;
   GemmArgs<double> a = args_in;
   constexpr int BM = MicroT<false, false>::BM, BN = MicroT<false, false>::BN;

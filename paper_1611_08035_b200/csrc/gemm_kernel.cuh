@@ -183,7 +183,9 @@ struct DmmaMicro {
   static constexpr int WTM = BM / WARPS_M, WTN = BN / WARPS_N;
   static constexpr int MI = WTM / 16, NI = WTN / 8;
   static constexpr bool REG_TRANSPOSE_B = false;
-  static constexpr bool HAS_KSPLIT = false;
+  // k split over a cluster: a lane's accumulators as MI*NI*4 64-bit words
+  static constexpr bool HAS_KSPLIT = true;
+  static constexpr int ACC_WORDS = MI * NI * 4;
   static_assert(WTM % 16 == 0 && WTN % 8 == 0 && BK % 16 == 0, "warp tile must be built from 16x8 fragments");
   // Fragment loads read either layout, so tiles are staged in their source layout.
   static constexpr Layout LA = TA ? KC : OC;
@@ -207,6 +209,14 @@ struct DmmaMicro {
       for (int ni = 0; ni < NI; ++ni)
 #pragma unroll
         for (int r = 0; r < 4; ++r) acc.c[mi][ni][r] = 0.0;
+  }
+  // word w of the accumulators as bits, and acc[w] += the double held in `bits` (one IEEE addition)
+  static __device__ __forceinline__ unsigned long long get_word(const Acc& acc, int w) {
+    return (unsigned long long)__double_as_longlong(acc.c[w / (NI * 4)][(w / 4) % NI][w % 4]);
+  }
+  static __device__ __forceinline__ void add_word(Acc& acc, int w, unsigned long long bits) {
+    double& c = acc.c[w / (NI * 4)][(w / 4) % NI][w % 4];
+    c = __dadd_rn(c, __longlong_as_double((long long)bits));
   }
 
   // One BK-deep slab: BK/4 k-steps of MI*NI independent mma.
@@ -374,15 +384,19 @@ struct SimtMicro {
     unsigned long long p[TM / 2][TN];
   };
   using Acc = typename std::conditional<PAIRS, AccPairs, AccScalar>::type;
-  static __device__ __forceinline__ unsigned long long& word(AccPairs& acc, int w) { return acc.p[w / TN][w % TN]; }
-  // a += b on both halves of a pair (two IEEE fp32 additions)
-  static __device__ __forceinline__ void add_pair(unsigned long long& a, unsigned long long b) {
+  static __device__ __forceinline__ unsigned long long get_word(const AccPairs& acc, int w) { return acc.p[w / TN][w % TN]; }
+  // acc[w] += b on both halves of a pair (two IEEE fp32 additions)
+  static __device__ __forceinline__ void add_word(AccPairs& acc, int w, unsigned long long b) {
+    unsigned long long& a = acc.p[w / TN][w % TN];
     float a0, a1, b0, b1;
     asm("mov.b64 {%0, %1}, %2;" : "=f"(a0), "=f"(a1) : "l"(a));
     asm("mov.b64 {%0, %1}, %2;" : "=f"(b0), "=f"(b1) : "l"(b));
     a0 = __fadd_rn(a0, b0), a1 = __fadd_rn(a1, b1);
     asm("mov.b64 %0, {%1, %2};" : "=l"(a) : "f"(a0), "f"(a1));
   }
+  // (scalar accumulators are never split: HAS_KSPLIT is false for them)
+  static __device__ __forceinline__ unsigned long long get_word(const AccScalar&, int) { return 0ull; }
+  static __device__ __forceinline__ void add_word(AccScalar&, int, unsigned long long) {}
 
   static __device__ __forceinline__ void zero(Acc& acc) {
     if constexpr (PAIRS) {
@@ -734,7 +748,7 @@ struct GemmKernel {
         __syncthreads();  // every warp has finished reading the ring
         if (blockIdx.z != 0) {
 #pragma unroll
-          for (int w = 0; w < Micro::ACC_WORDS; ++w) sAcc[w * NT + tid] = Micro::word(acc, w);
+          for (int w = 0; w < Micro::ACC_WORDS; ++w) sAcc[w * NT + tid] = Micro::get_word(acc, w);
         }
         cluster_sync_all();  // partial sums are visible across the cluster
         if (blockIdx.z == 0) {
@@ -742,7 +756,7 @@ struct GemmKernel {
             const uint32_t remote = cluster_map_shared(smem_u32(sAcc), (uint32_t)r);
 #pragma unroll
             for (int w = 0; w < Micro::ACC_WORDS; ++w)
-              Micro::add_pair(Micro::word(acc, w), ld_cluster_b64(remote + (uint32_t)((w * NT + tid) * 8)));
+              Micro::add_word(acc, w, ld_cluster_b64(remote + (uint32_t)((w * NT + tid) * 8)));
           }
         }
         cluster_sync_all();  // rank 0 has read everything: the other CTAs may leave

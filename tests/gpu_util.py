@@ -8,6 +8,9 @@ import torch
 from helpers import U
 from paper_1611_08035_b200 import synth
 
+GUARD = 1024       # guard-band elements on each side of every device operand (a multiple of 256 bytes)
+GUARD_BYTE = 0xA5  # as fp64/fp32 a large negative number no test produces
+
 TORCH_DT = {"d": torch.float64, "s": torch.float32, "z": torch.complex128, "z3": torch.complex128}
 
 
@@ -27,7 +30,8 @@ def run_and_check(b2, oracle, kind, transa, transb, m, n, k, alpha, beta, dist="
 
     Checks: every compared element within 2*k*u*S (complex: 2*(2k+4)*u*S per component, 3M 2*(3k+6)*u*S); bit-exact when
     expect_exact; padding rows of C and unsampled nothing-else untouched; A and B unchanged.
-    `offset` shifts every base pointer by that many elements (misaligned bases)."""
+    `offset` shifts every base pointer by that many elements (misaligned bases).  Every device operand sits
+    between guard bands that must come back untouched."""
     tdt = TORCH_DT[kind]
     (ra, ca), (rb, cb) = synth.operand_shapes(transa, transb, m, n, k)
     if lds is not None:
@@ -39,13 +43,20 @@ def run_and_check(b2, oracle, kind, transa, transb, m, n, k, alpha, beta, dist="
     A, lda, B, ldb, C, ldc = synth.gemm_inputs(transa, transb, m, n, k, dist, seed, tdt, lda, ldb, ldc, c_dist=c_dist)
     An, Bn, Cn = A.numpy(), B.numpy(), C.numpy()
 
+    guards = []
+
     def dev(x):
-        if offset:
-            buf = torch.empty(x.numel() + offset, dtype=x.dtype, device="cuda")
-            buf[offset:].copy_(x)
-            return buf, buf[offset:]
-        d = x.cuda()
-        return d, d
+        """Device copy of x bracketed by guard bands: GUARD elements of a fixed byte pattern directly before and
+        after it inside one allocation (the stand-in for a memory checker: a store before the first or past the
+        last element of an operand lands in a band and is seen below).  The front band is a multiple of 256 bytes,
+        so the operand keeps the alignment a fresh allocation has, then shifted by `offset` elements."""
+        count = x.numel()
+        buf = torch.empty(2 * GUARD + offset + count, dtype=x.dtype, device="cuda")
+        buf.view(torch.uint8).fill_(GUARD_BYTE)
+        body = buf[GUARD + offset:GUARD + offset + count]
+        body.copy_(x)
+        guards.append((buf, GUARD + offset, count))
+        return buf, body
 
     Ah, Ad = dev(A)
     Bh, Bd = dev(B)
@@ -74,6 +85,11 @@ def run_and_check(b2, oracle, kind, transa, transb, m, n, k, alpha, beta, dist="
     assert b2.b2_device_status() == 0, "a device-side wait timed out"
     torch.cuda.synchronize()
     got = Cd.cpu().numpy()
+    for buf, start, count in guards:
+        raw = buf.view(torch.uint8)
+        es = buf.element_size()
+        assert bool((raw[:start * es] == GUARD_BYTE).all()), "bytes before an operand were written"
+        assert bool((raw[(start + count) * es:] == GUARD_BYTE).all()), "bytes behind an operand were written"
     assert torch.equal(Ad.cpu().view(torch.uint8), A.view(torch.uint8)), "A was modified"
     assert torch.equal(Bd.cpu().view(torch.uint8), B.view(torch.uint8)), "B was modified"
 

@@ -280,6 +280,38 @@ def test_sgemm_k_split_over_cluster(b2, oracle):
     assert all(torch.equal(outs[0].view(torch.uint8), o.view(torch.uint8)) for o in outs[1:])
 
 
+def test_dgemm_k_split_over_cluster(b2, oracle):
+    """The fp64 tensor-core kernels with the k-loop of every tile split over a cluster of two or four CTAs
+    (requested as variant + 256*s): ragged sizes, all transposes, padded and aligned leading dimensions, a k too
+    short to give every CTA a slab; exact on integer data, within the bound otherwise, the same bits on every
+    run; variants that cannot split decline without writing."""
+    names = [b2.b2_variant_name(0, v) for v in range(nvariants(b2, "d"))]
+    for v, name in enumerate(names):
+        for split in (2, 4):
+            if "tma" in name or "dfma" in name:
+                C = torch.ones(64 * 64, dtype=torch.float64, device="cuda")
+                rc = b2.b2_dgemm("N", "N", 64, 64, 64, 1.0, C, 64, C, 64, 0.0, C.clone(), 64, variant=v + 256 * split,
+                                 check=False)
+                assert rc == 1004, f"{name} accepted a k split"
+                continue
+            for ta, tb in TRANS:
+                run_and_check(b2, oracle, "d", ta, tb, 333, 270, 145, 0.7, -0.3, seed=v, pad=True,
+                              variant=v + 256 * split)
+                run_and_check(b2, oracle, "d", ta, tb, 300, 260, 136, 1.5, 0.5, dist="int9", seed=v,
+                              variant=v + 256 * split, expect_exact=True)
+            run_and_check(b2, oracle, "d", "N", "N", 130, 70, 33, 1.0, 0.0, seed=3, variant=v + 256 * split)  # 3 slabs
+            run_and_check(b2, oracle, "d", "N", "N", 65, 129, 7, 0.7, -0.3, seed=4, variant=v + 256 * split)   # 1 slab
+    assert b2.b2_dgemm("N", "N", 64, 64, 64, 1.0, C, 64, C, 64, 0.0, C.clone(), 64, variant=2 + 256 * 3,
+                       check=False) == 1004
+    A, lda, B, ldb, C, ldc = synth.gemm_inputs("T", "N", 1001, 999, 1003, "uniform", 55, torch.float64)
+    outs = []
+    for _ in range(3):
+        Cd = C.cuda()
+        b2.b2_dgemm("T", "N", 1001, 999, 1003, 0.7, A.cuda(), lda, B.cuda(), ldb, -0.3, Cd, ldc, variant=2 + 512)
+        outs.append(Cd.cpu())
+    assert all(torch.equal(outs[0].view(torch.uint8), o.view(torch.uint8)) for o in outs[1:])
+
+
 # ---- complex 4M ------------------------------------------------------------------------------------
 
 def test_zgemm4m_small_full_all_transposes(b2, oracle):
