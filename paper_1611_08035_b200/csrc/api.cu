@@ -23,6 +23,8 @@ int launch_f64_v6(const GemmArgs<double>&, bool, bool, bool, cudaStream_t);
 int launch_f64_t32(const GemmArgs<double>&, bool, bool, bool, cudaStream_t);
 int launch_f64_tma_t32(const GemmArgs<double>&, bool, bool, bool, cudaStream_t);
 int launch_f64_w8(const GemmArgs<double>&, bool, bool, bool, cudaStream_t);
+int launch_f64_ws_64x64(const GemmArgs<double>&, bool, bool, bool, cudaStream_t);
+int launch_f64_ws_64x64_direct(const GemmArgs<double>&, bool, bool, bool, cudaStream_t);
 int launch_f32_v0(const GemmArgs<float>&, bool, bool, bool, cudaStream_t);
 int launch_f32_v1(const GemmArgs<float>&, bool, bool, bool, cudaStream_t);
 int launch_f32_v2(const GemmArgs<float>&, bool, bool, bool, cudaStream_t);
@@ -43,10 +45,13 @@ const VariantInfo kF64Info[] = {
     {"dmma_32x32x16_s3", "dmma", 32, 32, 16, 3, 128, 6, 0.80},
     {"dmma_tma_32x32x16_s3", "dmma_tma", 32, 32, 16, 3, 128, 6, 0.80},
     {"dmma_w8_64x64x16_s3", "dmma", 64, 64, 16, 3, 256, 3, 0.92},
+    {"dmma_ws_3x64x64x16_s3", "dmma_ws", 64, 64, 16, 3, 512, 1, 0.95},
+    {"dmma_ws_direct_3x64x64x16_s3", "dmma_ws", 64, 64, 16, 3, 512, 1, 0.95},
 };
 const LaunchFn<double> kF64Launch[] = {launch_f64_v0, launch_f64_v1, launch_f64_v2, launch_f64_v3,
                                        launch_f64_v4, launch_f64_v5, launch_f64_v6, launch_f64_t32,
-                                       launch_f64_tma_t32, launch_f64_w8};
+                                       launch_f64_tma_t32, launch_f64_w8, launch_f64_ws_64x64,
+                                       launch_f64_ws_64x64_direct};
 const VariantInfo kF32Info[] = {
     {"ffma2_t16x8_128x128x16_s3", "ffma2", 128, 128, 16, 3, 128, 2, 0.782, 16, 8, 3500.0, 11.0},
     {"ffma2_128x64x16_s4", "ffma2", 128, 64, 16, 4, 128, 3, 0.795, 8, 8, 0.0, 5.8, true},
@@ -142,7 +147,8 @@ int choose_variant(int64_t m, int64_t n, int64_t k, bool aligned, int64_t batch 
   TileChoice cand[16];
   for (int v = 0; v < count && v < 16; ++v) {
     const VariantInfo& vi = variant_info_t<T>(v);
-    const bool comparison_only = strcmp(vi.micro, "dfma") == 0 || strcmp(vi.micro, "ffma") == 0;
+    const bool comparison_only = strcmp(vi.micro, "dfma") == 0 || strcmp(vi.micro, "ffma") == 0 ||
+                                 strcmp(vi.micro, "dmma_ws") == 0;
     const bool needs_alignment = strcmp(vi.micro, "dmma_tma") == 0;
     double eff = vi.efficiency;
     // Unaligned operands are staged in 8- or 4-byte pieces: twice to four times the staging instructions, which

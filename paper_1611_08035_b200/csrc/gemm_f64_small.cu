@@ -5,6 +5,6 @@ namespace b2 {
 template <bool TA, bool TB>
 using MicroF64T32 = DmmaMicro<32, 32, 16, 2, 2, TA, TB>;
 int launch_f64_t32(const GemmArgs<double>& a, bool ta, bool tb, bool aligned, cudaStream_t s) {
-  return VariantLauncher<MicroF64T32, 3, 6>::launch(a, ta, tb, aligned, s);
+  return VariantLauncher<MicroF64T32, 3, 7>::launch(a, ta, tb, aligned, s);
 }
 }  // namespace b2

@@ -30,6 +30,8 @@ EncodeFn encode_fn() {
   return fn;
 }
 
+}  // namespace
+
 // 2-D fp64 tensor map of a column-major matrix (rows contiguous) with the given box.
 bool make_map(CUtensorMap* map, const double* base, int64_t rows, int64_t cols, int64_t ld, int box_inner,
               int box_outer) {
@@ -57,6 +59,8 @@ int* status_pointer() {
   }
   return cached;
 }
+
+namespace {
 
 template <class Kernel, int MIN_CTAS, bool TA, bool TB>
 int launch_tma_one(const GemmArgs<double>& a, cudaStream_t stream) {

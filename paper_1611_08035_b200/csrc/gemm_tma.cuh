@@ -44,6 +44,19 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
       : "memory");
   return done != 0;
 }
+// Non-blocking test of a phase (try_wait may suspend the thread for a while; a thread that polls several
+// barriers in turn must not).
+__device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t done;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(done)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return done != 0;
+}
 // Bounded wait: false when the phase did not complete within limit_ns nanoseconds of wall time.  The bound is a
 // time (the global nanosecond timer), not a number of polls, because one try_wait may itself block for an
 // implementation-defined interval.  A wait that succeeds at once never reads the timer; after that the timer is
@@ -76,6 +89,32 @@ __device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* m
       "r"(smem_u32(bar))
       : "memory");
 }
+
+// ---- untiled bulk copies (both addresses 16-byte aligned, size a multiple of 16 bytes) ---------------------
+// global -> shared, completion counted on `bar`
+__device__ __forceinline__ void bulk_load(void* smem_dst, const void* gmem_src, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                   smem_u32(smem_dst)),
+               "l"(gmem_src), "r"(bytes), "r"(smem_u32(bar))
+               : "memory");
+}
+// shared -> global, tracked by the issuing thread's bulk async-groups
+__device__ __forceinline__ void bulk_store(void* gmem_dst, const void* smem_src, uint32_t bytes) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gmem_dst), "r"(smem_u32(smem_src)),
+               "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// all of this thread's bulk stores have read their shared-memory source / have completed
+__device__ __forceinline__ void bulk_wait_read_all() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
+// ---- host helpers shared by the TMA-staged kernels (defined in gemm_f64_tma.cu) ------------------
+// 2-D fp64 tensor map of a column-major matrix (rows contiguous, leading dimension ld) with the given box.
+bool make_map(CUtensorMap* map, const double* base, int64_t rows, int64_t cols, int64_t ld, int box_inner,
+              int box_outer);
+// Device address (on the current device) of the status word that bounded waits write; nullptr on failure.
+int* status_pointer();
 
 // ---- the kernel ------------------------------------------------------------------------------
 template <class Micro, int STAGES, bool TA, bool TB>

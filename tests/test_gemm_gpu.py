@@ -10,7 +10,7 @@ import numpy as np
 import pytest
 import torch
 
-from gpu_util import run_and_check, sample_columns
+from gpu_util import run_and_check, sample_columns, staged_by_tma
 from paper_1611_08035_b200 import synth
 
 pytestmark = pytest.mark.gpu
@@ -74,7 +74,7 @@ def test_rank_k_update_whole_matrix_every_staging(b2, oracle, k):
     for v, name in enumerate(names):
         if "dmma" not in name:
             continue
-        for rep in range(3 if "tma" in name else 1):
+        for rep in range(3 if staged_by_tma(name) else 1):
             Cd = C.clone()
             b2.b2_dgemm("N", "N", m, n, k, -1.0, A, lda, B, ldb, 1.0, Cd, ldc, variant=v)
             assert b2.b2_device_status() == 0
@@ -137,7 +137,7 @@ def test_all_variants_multi_tile_ragged(b2, oracle, kind):
 def test_tma_variants_aligned_ragged_shapes(b2, oracle):
     """The TMA-staged variants on shapes with ragged m, n and k (edge tiles and the partial last slab are
     zero-filled by the hardware), even leading dimensions for A and B, an odd one for C."""
-    tma = [v for v in range(nvariants(b2, "d")) if "tma" in b2.b2_variant_name(0, v)]
+    tma = [v for v in range(nvariants(b2, "d")) if staged_by_tma(b2.b2_variant_name(0, v))]
     assert len(tma) >= 3
     for v in tma:
         for ta, tb in TRANS:
@@ -288,7 +288,7 @@ def test_dgemm_k_split_over_cluster(b2, oracle):
     names = [b2.b2_variant_name(0, v) for v in range(nvariants(b2, "d"))]
     for v, name in enumerate(names):
         for split in (2, 4):
-            if "tma" in name or "dfma" in name:
+            if staged_by_tma(name) or "dfma" in name:
                 C = torch.ones(64 * 64, dtype=torch.float64, device="cuda")
                 rc = b2.b2_dgemm("N", "N", 64, 64, 64, 1.0, C, 64, C, 64, 0.0, C.clone(), 64, variant=v + 256 * split,
                                  check=False)

@@ -14,7 +14,7 @@ import numpy as np
 import pytest
 import torch
 
-from gpu_util import sample_columns
+from gpu_util import sample_columns, staged_by_tma
 from paper_1611_08035_b200 import synth
 
 pytestmark = pytest.mark.gpu
@@ -48,7 +48,7 @@ def test_fp64_every_tensor_core_variant_same_bits(b2, oracle, size):
     for v, name in list(enumerate(names)) + [(None, "auto")]:
         if v is not None and "dmma" not in name:
             continue
-        for rep in range(3 if "tma" in name else 1):
+        for rep in range(3 if staged_by_tma(name) else 1):
             Cd = C.clone()
             b2.b2_dgemm("N", "N", m, n, k, 1.5, A, lda, B, ldb, 0.5, Cd, ldc, variant=v)
             assert b2.b2_device_status() == 0
@@ -69,7 +69,7 @@ def test_fp64_transposed_staging_same_bits_4096(b2, oracle, ta, tb):
         name = b2.b2_variant_name(0, v)
         if "dmma" not in name or "32x32" in name:
             continue
-        for rep in range(2 if "tma" in name else 1):
+        for rep in range(2 if staged_by_tma(name) else 1):
             Cd = C.clone()
             b2.b2_dgemm(ta, tb, m, n, k, 1.5, A, lda, B, ldb, 0.5, Cd, ldc, variant=v)
             assert b2.b2_device_status() == 0
