@@ -352,15 +352,30 @@ int b2_pipe_probe(int kind, int threads_per_cta, int ctas, int64_t iters, void* 
  * b2_model_predict_variant: the Section 4 estimate applied to one sub-partition of a B200 SM
  *   (pipelines: issue, FP64 FMA, FP64 tensor, FP32 FMA, shared-memory wavefronts; rates from
  *   b2_pipe_probe) for kernel variant `variant` of `dtype`.  Stores the predicted fraction of the
- *   arithmetic pipe's peak in *fraction and, when json_out is not NULL, a JSON object with the
- *   jobs per pipeline per rank-1 update, the clocks each pipeline needs, the prediction and the
- *   measured steady-state fraction (HOST buffer of cap bytes).  Returns 0, -1/-2/-3 for a bad
+ *   arithmetic pipe's peak in *fraction: min(pipeline estimate, L2 feed) x latency coverage (the
+ *   paper's sizing rule of Section 4 read as Little's law over all warps of a scheduler).  When
+ *   json_out is not NULL it receives a JSON object with the jobs per pipeline per rank-1 update, the
+ *   clocks each pipeline needs, the three factors, registers and resident CTAs, the prediction and
+ *   the measured steady-state fraction (HOST buffer of cap bytes).  Returns 0, -1/-2/-3 for a bad
  *   dtype / variant / null fraction, B2_ERR_WORKSPACE when cap is too small.
  */
 double b2_model_throughput(int npipes, const double* rate, const double* jobs);
 double b2_model_stalled_throughput(double jobs, int n_dependent, double latency);
 int b2_model_register_updates(int r_total, int mr, int nr, int v, int r_a, int r_r, int* n_updates);
 int b2_model_predict_variant(int dtype, int variant, double* fraction, char* json_out, size_t cap);
+/*
+ * b2_model_enumerate: Section 5.1 ("A Work Flow for Kernel Generation": enumerate the ways to compute the outer
+ *   product, estimate each with the model of Section 4, keep the best) for the SM.  Candidates are micro-kernel
+ *   kind (dtype 0: DMMA, DFMA; dtype 1: packed-pair and scalar FFMA) x warp tile x warp grid of a CTA x ring
+ *   stages; a candidate is kept when it fits the register limit of Section 5 restated for a thread (accumulators
+ *   + R_A + at least two unit updates' fragments <= 255, and the SM's register file and shared memory for at
+ *   least one CTA; the limits are queried from the current device, B200 values without one).  Each is scored
+ *   with predicted fraction = min(pipeline estimate, L2 feed) x latency coverage at the residency it reaches.
+ *   json_out (HOST, cap bytes) receives {"dtype", "candidates", "ranked": [...]} with the best `top` candidates in
+ *   rank order and, whatever their rank, the candidates that exist as variants of this library ("built_as").
+ *   Returns 0, -1 / -2 / -3 for a bad dtype / top <= 0 / null buffer, B2_ERR_WORKSPACE when cap is too small.
+ */
+int b2_model_enumerate(int dtype, int top, char* json_out, size_t cap);
 
 /* Static, NUL-terminated text for a return value of any call above. */
 const char* b2_strerror(int status);

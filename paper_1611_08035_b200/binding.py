@@ -77,6 +77,7 @@ _SIGNATURES = {
     "b2_model_stalled_throughput": (c_double, [c_double, c_int, c_double]),
     "b2_model_register_updates": (c_int, [c_int, c_int, c_int, c_int, c_int, c_int, ctypes.POINTER(c_int)]),
     "b2_model_predict_variant": (c_int, [c_int, c_int, ctypes.POINTER(c_double), c_char_p, c_size_t]),
+    "b2_model_enumerate": (c_int, [c_int, c_int, c_char_p, c_size_t]),
     "b2_strerror": (c_char_p, [c_int]),
     "b2_version": (c_char_p, []),
 }
@@ -354,6 +355,13 @@ def b2_model_register_updates(r_total, mr, nr, v, r_a, r_r) -> int:
     out = c_int(0)
     _check("b2_model_register_updates", lib().b2_model_register_updates(r_total, mr, nr, v, r_a, r_r, ctypes.byref(out)))
     return out.value
+
+
+def b2_model_enumerate(dtype: int, top: int = 16) -> str:
+    """Ranked candidate micro-kernels/tiles of the pipeline model as a JSON string (host-only call)."""
+    buf = ctypes.create_string_buffer(1 << 16)
+    _check("b2_model_enumerate", lib().b2_model_enumerate(dtype, top, buf, len(buf)))
+    return buf.value.decode()
 
 
 def b2_model_predict_variant(dtype: int, variant: int):

@@ -9,6 +9,7 @@
 #include "b2gemm.h"
 #include "entry.h"
 #include "gemm_launch.cuh"
+#include "queue_model.h"
 #include "select.h"
 
 namespace b2 {
@@ -31,7 +32,11 @@ int launch_f32_v2(const GemmArgs<float>&, bool, bool, bool, cudaStream_t);
 int launch_f32_v3(const GemmArgs<float>&, bool, bool, bool, cudaStream_t);
 int launch_f32_s32(const GemmArgs<float>&, bool, bool, bool, cudaStream_t);
 
+model::SmPrediction predict_variant(int dtype, int variant);  // model_api.cu
+
 namespace {
+
+constexpr double kModelTrust = 0.05;
 
 // name, micro-kernel, BM, BN, BK, stages, threads, resident CTAs per SM, measured steady-state efficiency
 const VariantInfo kF64Info[] = {
@@ -42,9 +47,9 @@ const VariantInfo kF64Info[] = {
     {"dmma_tma_64x64x16_s3", "dmma_tma", 64, 64, 16, 3, 128, 4, 0.97},
     {"dmma_tma_128x64x16_s3", "dmma_tma", 128, 64, 16, 3, 128, 2, 0.945},
     {"dmma_tma_128x128x16_s4", "dmma_tma", 128, 128, 16, 4, 256, 1, 0.95},
-    {"dmma_32x32x16_s3", "dmma", 32, 32, 16, 3, 128, 6, 0.80},
+    {"dmma_32x32x16_s3", "dmma", 32, 32, 16, 3, 128, 7, 0.80, 8, 8, 0.0, 7.0, true},
     {"dmma_tma_32x32x16_s3", "dmma_tma", 32, 32, 16, 3, 128, 6, 0.80},
-    {"dmma_w8_64x64x16_s3", "dmma", 64, 64, 16, 3, 256, 3, 0.92},
+    {"dmma_w8_64x64x16_s3", "dmma_w8", 64, 64, 16, 3, 256, 3, 0.91},
     {"dmma_ws_3x64x64x16_s3", "dmma_ws", 64, 64, 16, 3, 512, 1, 0.95},
     {"dmma_ws_direct_3x64x64x16_s3", "dmma_ws", 64, 64, 16, 3, 512, 1, 0.95},
 };
@@ -57,7 +62,7 @@ const VariantInfo kF32Info[] = {
     {"ffma2_128x64x16_s4", "ffma2", 128, 64, 16, 4, 128, 3, 0.795, 8, 8, 0.0, 5.8, true},
     {"ffma2_64x64x16_s4", "ffma2", 64, 64, 16, 4, 64, 6, 0.64},
     {"ffma_128x64x16_s4", "ffma", 128, 64, 16, 4, 128, 4, 0.70},
-    {"ffma2_t4_32x32x16_s4", "ffma2", 32, 32, 16, 4, 64, 8, 0.40, 4, 4},
+    {"ffma2_t4_32x32x16_s4", "ffma2", 32, 32, 16, 4, 64, 8, 0.40, 4, 4, 0.0, 7.0, true},
 };
 const LaunchFn<float> kF32Launch[] = {launch_f32_v0, launch_f32_v1, launch_f32_v2, launch_f32_v3, launch_f32_s32};
 
@@ -147,10 +152,17 @@ int choose_variant(int64_t m, int64_t n, int64_t k, bool aligned, int64_t batch 
   TileChoice cand[16];
   for (int v = 0; v < count && v < 16; ++v) {
     const VariantInfo& vi = variant_info_t<T>(v);
+    // measured counterparts, never chosen automatically: the FMA micro-kernels on fp64 / scalar fp32, the
+    // eight-warp 64 x 64 tile (slower than the four-warp one wherever it was measured) and the persistent kernel
     const bool comparison_only = strcmp(vi.micro, "dfma") == 0 || strcmp(vi.micro, "ffma") == 0 ||
-                                 strcmp(vi.micro, "dmma_ws") == 0;
+                                 strcmp(vi.micro, "dmma_ws") == 0 || strcmp(vi.micro, "dmma_w8") == 0;
     const bool needs_alignment = strcmp(vi.micro, "dmma_tma") == 0;
-    double eff = vi.efficiency;
+    // Steady-state fraction of the arithmetic pipe at full residency: the pipeline model's prediction (Section 4
+    // estimate x latency coverage x barrier stall, queue_model.h).  The table's measured value is the recorded check
+    // of that prediction; it replaces it only where the two are more than kModelTrust apart (fp32 tiles whose
+    // element-wise transposing copies the model does not price, the 32 x 32 cp.async tile).
+    const model::SmPrediction pr = predict_variant(sizeof(T) == 8 ? B2_F64 : B2_F32, v);
+    double eff = (pr.feasible && fabs(pr.fraction - vi.efficiency) <= kModelTrust) ? pr.fraction : vi.efficiency;
     // Unaligned operands are staged in 8- or 4-byte pieces: twice to four times the staging instructions, which
     // weigh the more the smaller the tile (staging work per multiply-add goes with (BM+BN)/(BM*BN)); measured on
     // the 1001 x 999 x 1003 problem with odd leading dimensions.
@@ -185,6 +197,10 @@ int choose_variant(int64_t m, int64_t n, int64_t k, bool aligned, int64_t batch 
         // with fewer tiles than a quarter of the SMs the 32 x 32 tile is the better tool (512^3 TN: 18.5 us against 24.4)
         const int64_t tiles = ((m + vi.bm - 1) / vi.bm) * ((n + vi.bn - 1) / vi.bn) * (batch < 1 ? 1 : batch);
         if (4 * tiles < sms) break;
+        // small tiles that fill an SM with six or more CTAs gain from a split only while the tiles themselves are
+        // fewer than about one per SM (measured: 32 x 32 tiles, both data types, split better at 256^3 and 384^3,
+        // 64 and 144 tiles, worse at 512^3, 256 tiles)
+        if (vi.ctas_per_sm >= 6 && 4 * tiles > 5 * (int64_t)sms) break;
         const int64_t k_part = (slabs + split - 1) / split * vi.bk;
         TileChoice c = cand[v];
         // reduction: two cluster barriers and, for the first CTA, the other CTAs' accumulators through

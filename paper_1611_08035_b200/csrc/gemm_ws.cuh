@@ -80,6 +80,8 @@ struct GemmWsKernel {
   static constexpr int C_PITCH = BM + 2;
   static constexpr uint32_t CBUF_BYTES = STAGE_C ? BN * C_PITCH * 8 : 0;
   static constexpr uint32_t COL_BYTES = BM * 8;
+  // old C values of a tile are requested in this many batches (one: all 32 values of a thread in flight at once)
+  static constexpr int C_BATCHES = CONSUMER_REGS >= 152 ? 1 : 2;
   static constexpr size_t RING_BYTES = (size_t)GROUPS * GSTAGES * STAGE_BYTES;
   static constexpr int NBARS = 2 * GROUPS * GSTAGES + 3 * GROUPS;  // full, empty; cdone, stagger, sfree
   static constexpr size_t BAR_OFFSET = RING_BYTES + CBUF_BYTES;
@@ -221,6 +223,16 @@ struct GemmWsKernel {
     for (int i = g, u = 0; i < my_tiles && ok; i += GROUPS, ++u) {
       int m0, n0;
       tile_origin(i, m0, n0);
+      // beta != 0: pull the tile's old C values towards L2 while the k-loop runs
+      if (use_beta) {
+        const int m_valid = (int)min((int64_t)BM, p.m - m0), n_valid = (int)min((int64_t)BN, p.n - n0);
+        constexpr int LINE = 16, LPC = BM / LINE;  // 128-byte lines per tile column
+        for (int c = ltid; c < BN * LPC; c += GT) {
+          const int col = c / LPC, row = (c % LPC) * LINE;
+          if (col < n_valid && row < m_valid)
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(p.C + (int64_t)(n0 + col) * p.ldc + m0 + row));
+        }
+      }
       typename Micro::Acc acc;
       Micro::zero(acc);
       for (int kt = 0; kt < KT; ++kt, ++cnt) {
@@ -251,10 +263,10 @@ struct GemmWsKernel {
       const bool staged = STAGE_C && c_vec_ok && (int64_t)m0 + BM <= p.m && (int64_t)n0 + BN <= p.n;
       if (staged) {
         T* cfrag = p.C + (int64_t)(n0 + fcol) * p.ldc + m0 + frow;
-        // results into the accumulator registers; the old values are fetched in two batches
+        // results into the accumulator registers; the old values are fetched in C_BATCHES batches
 #pragma unroll
-        for (int half = 0; half < 2; ++half) {
-          constexpr int NH = Micro::NI / 2;
+        for (int half = 0; half < C_BATCHES; ++half) {
+          constexpr int NH = Micro::NI / C_BATCHES;
           double2 old[Micro::MI][NH][2];
           if (use_beta) {
 #pragma unroll

@@ -62,6 +62,13 @@ inline void sm_rates(double (&rate)[NPIPES]) {
 
 enum MicroKind { MK_DMMA = 0, MK_DFMA = 1, MK_FFMA = 2, MK_FFMA2 = 3 };
 
+// Scalar 32-bit multiply-adds with three distinct register sources issue below one per clock when the compiler,
+// not the programmer, places the operands (register-bank conflicts the packed 64-bit operands do not have); the
+// same holds for FP64 multiply-adds on their pipe.  Slots per instruction, fitted to the two comparison kernels
+// (scalar FFMA 0.70, DFMA 0.73 of peak); the tensor-core and packed-pair kernels carry no such factor.
+constexpr double kScalarFmaSlots = 1.30;
+constexpr double kDfmaSlots = 1.37;
+
 // Jobs per pipeline for one rank-1 update (one k) of one warp's tile.
 //   wtm x wtn     the warp's block of C (DMMA: 16x8 fragments; FMA kinds: 8 lanes x 4 lanes of tm x tn blocks,
 //                 8 x 8 -> 64 x 32, 16 x 8 -> 128 x 32, 4 x 4 -> 32 x 16)
@@ -89,14 +96,17 @@ inline WarpMix warp_mix(int kind, int wtm, int wtn, int staging_per_slab, int sl
     const double loads = (tm + tn) / (f64 ? 2.0 : 4.0);  // tm + tn operand values per lane in 16-byte loads
     m.jobs[LSU] = loads;                         // lanes of a warp share operands: one wavefront per load
     if (kind == MK_DFMA) {
-      m.jobs[FP64] = fma;
+      m.jobs[FP64] = fma * kDfmaSlots;
       m.jobs[ISSUE] = fma + loads + overhead;
     } else if (kind == MK_FFMA) {
       m.jobs[FP32] = fma;
-      m.jobs[ISSUE] = fma + loads + overhead;
+      m.jobs[ISSUE] = fma * kScalarFmaSlots + loads + overhead;
     } else {
-      m.jobs[FP32] = fma;                        // 32 packed instructions, two jobs each
-      m.jobs[ISSUE] = fma / 2.0 + loads + tn + overhead;  // plus the moves that duplicate the tn values of b
+      // 32 packed instructions, two jobs each, plus the moves that copy each of the tn values of b into both halves
+      // of a pair: two 32-bit moves per value, executed on the same FP32 pipe (the profiler puts them at a fifth of
+      // that pipe's activity in the 8 x 8 kernel: 16 of 80 jobs)
+      m.jobs[FP32] = fma + 2.0 * tn;
+      m.jobs[ISSUE] = fma / 2.0 + loads + 2.0 * tn + overhead;
     }
   }
   return m;
@@ -111,6 +121,118 @@ inline double predicted_fraction(const WarpMix& m, bool fp64_data) {
   const double peak = fp64_data ? 16.0 : 32.0;
   const double f = lam * m.fma_per_k / peak;
   return f > 1.0 ? 1.0 : f;
+}
+
+// ---- latency coverage (Section 4, "Dealing with dependencies across pipelines") ------------------------
+// The paper sizes mr x nr so that the multiply-adds of one outer product are independent and cover the pipeline's
+// latency; when they do not, the dependent instructions wait (W = L + n*k).  On an SM the instructions that can
+// cover a pipeline's latency are the independent arithmetic instructions of ALL warps resident on a scheduler:
+// I = warps per scheduler x independent instructions per unit update.  By Little's law the pipeline is kept full
+// once I exceeds latency x rate; the smooth form 1 - exp(-I / I0) is fitted to one measured point of the tensor
+// pipe (the TMA-staged 32 x 32 tile: six CTAs of four warps, two tensor instructions per warp and k-step, I = 12,
+// 0.80 of peak -> I0 = 7.5) and used for every pipeline.
+constexpr double kCoverageI0 = 7.5;
+// The stall term itself (W = L + n*k): kernels staged with cp.async pass one CTA-wide barrier per slab, at which
+// every warp of the CTA waits for the slowest and for the first fragments of the new slab: n = 1 dependent step
+// of k = kBarrierStallClks per slab, which the other CTAs resident on the SM cover in proportion to their number
+// (fitted to the one-CTA 128 x 128 DMMA kernel, 0.87 of peak; the FMA pipes, whose instructions return in a few
+// clocks instead of the tensor pipe's tens, refill sooner: fitted to the scalar FFMA kernel).  Kernels fed through
+// mbarriers by the tensor memory accelerator have no such step.
+constexpr double kBarrierStallClksTensor = 250.0;
+constexpr double kBarrierStallClksFma = 30.0;
+
+inline double latency_coverage(double independent_in_flight) {
+  return independent_in_flight <= 0.0 ? 0.0 : 1.0 - exp(-independent_in_flight / kCoverageI0);
+}
+
+// Limits of one SM that bound a candidate (queried from the device by the caller; B200 values as defaults).
+struct SmLimits {
+  int regs_per_sm = 65536;
+  int max_regs_per_thread = 255;
+  int smem_per_sm = 233472;  // bytes usable by CTAs
+  int max_warps_per_sm = 64;
+  int max_ctas_per_sm = 32;
+  double l2_feed_bytes_per_clk = 32.0;  // sustainable L2 -> shared-memory feed per SM
+};
+
+// A candidate micro-kernel/tile: kind, the warp's block of C, the warp grid of a CTA, slab depth and ring stages.
+struct SmCandidate {
+  int kind;              // MicroKind
+  int wtm, wtn;          // warp tile
+  int warps_m, warps_n;  // warps of a CTA along m and n
+  int bk, stages;
+  bool tma;              // operand slabs arrive by the tensor memory accelerator through mbarriers (no CTA-wide barrier)
+};
+
+struct SmPrediction {
+  bool feasible;        // fits registers and shared memory with at least two unit updates of fragments in flight
+  int bm, bn, threads;
+  int acc_regs, frag_regs, regs_per_thread;  // accumulators, fragments of one unit update, total (double-buffered)
+  int n_updates;        // Section 5: floor((R_thread - accumulators - R_A) / R_R), unit updates of fragments that fit
+  int smem_bytes;       // ring of `stages` slabs
+  int ctas_per_sm;
+  double pipe_fraction; // Section 4 estimate: min over pipelines, as a fraction of the arithmetic pipe's peak
+  double feed_fraction; // what the L2 -> shared-memory feed allows for this tile's bytes per multiply-add
+  double coverage;      // latency coverage at full residency
+  double stall;         // L / (L + n*k): the barrier stall of cp.async-staged kernels (1 for TMA-staged ones)
+  double fraction;      // product: the predicted fraction of peak
+};
+
+constexpr int kAddressRegs = 24;  // R_A: addresses, loop counters, barrier state
+
+inline SmPrediction predict(const SmCandidate& c, const SmLimits& lim, int elem_bytes) {
+  SmPrediction r = {};
+  const int w = elem_bytes / 4;  // 32-bit registers per value
+  r.bm = c.wtm * c.warps_m, r.bn = c.wtn * c.warps_n, r.threads = 32 * c.warps_m * c.warps_n;
+  r.acc_regs = c.wtm * c.wtn * w / 32;
+  double indep;  // independent arithmetic instructions of a warp per unit update
+  if (c.kind == MK_DMMA) {
+    const int mi = c.wtm / 16, ni = c.wtn / 8;
+    r.frag_regs = (2 * mi + ni) * w;  // a0, a1 per row block, b0 per column block
+    indep = mi * ni;
+  } else {
+    const int tm = c.wtm / 8, tn = c.wtn / 4;
+    r.frag_regs = (tm + tn) * w;
+    indep = (c.kind == MK_FFMA2) ? tm * tn / 2.0 : tm * tn;
+  }
+  // Section 5 restated for a thread: the register limit leaves room for N unit updates' worth of fragments;
+  // software pipelining needs two (the next unit update's fragments are loaded while the current one is multiplied).
+  r.n_updates = (lim.max_regs_per_thread - r.acc_regs - kAddressRegs) / (r.frag_regs > 0 ? r.frag_regs : 1);
+  r.regs_per_thread = r.acc_regs + 2 * r.frag_regs + kAddressRegs;
+  const int regs_alloc = (r.regs_per_thread + 7) / 8 * 8;
+  // ring: BK x (BM + BN) values per slab plus a few values of padding per line
+  r.smem_bytes = c.stages * c.bk * (r.bm + r.bn + 8) * elem_bytes;
+  const int by_regs = lim.regs_per_sm / (r.threads * regs_alloc);
+  const int by_smem = lim.smem_per_sm / (r.smem_bytes + 1024);
+  const int by_warps = lim.max_warps_per_sm / (r.threads / 32);
+  int ctas = by_regs < by_smem ? by_regs : by_smem;
+  if (by_warps < ctas) ctas = by_warps;
+  if (lim.max_ctas_per_sm < ctas) ctas = lim.max_ctas_per_sm;
+  r.ctas_per_sm = ctas;
+  r.feasible = r.n_updates >= 2 && ctas >= 1 && r.regs_per_thread <= lim.max_regs_per_thread && c.wtm > 0 && c.wtn > 0;
+  if (!r.feasible) return r;
+  const int staging = (r.bm + r.bn) * c.bk * elem_bytes / 16 / r.threads;
+  const WarpMix mix = warp_mix(c.kind, c.wtm, c.wtn, staging > 0 ? staging : 1, c.bk);
+  r.pipe_fraction = predicted_fraction(mix, elem_bytes == 8);
+  const double fma_per_clk = elem_bytes == 8 ? 64.0 : 128.0;
+  const double bytes_per_fma = (double)(r.bm + r.bn) * elem_bytes / ((double)r.bm * r.bn);
+  const double feed = lim.l2_feed_bytes_per_clk / (fma_per_clk * bytes_per_fma);
+  r.feed_fraction = feed > 1.0 ? 1.0 : feed;
+  const double warps_per_scheduler = ctas * (r.threads / 32) / 4.0;
+  r.coverage = latency_coverage(warps_per_scheduler * indep);
+  // clocks the slowest pipeline needs for one slab of one warp, at the SM's full rate for this warp's share
+  double rate[NPIPES];
+  sm_rates(rate);
+  double slab_clks = 0.0;
+  for (int i = 0; i < NPIPES; ++i) {
+    const double t = mix.jobs[i] / rate[i] * c.bk;
+    if (t > slab_clks) slab_clks = t;
+  }
+  const double k_stall = (c.kind == MK_DMMA ? kBarrierStallClksTensor : kBarrierStallClksFma) / ctas;
+  r.stall = c.tma ? 1.0 : stalled_throughput(slab_clks, 1, k_stall) * slab_clks;  // L / (L + n*k)
+  const double bound = r.pipe_fraction < r.feed_fraction ? r.pipe_fraction : r.feed_fraction;
+  r.fraction = bound * r.coverage * r.stall;
+  return r;
 }
 
 }  // namespace model

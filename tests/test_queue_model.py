@@ -120,27 +120,97 @@ def test_library_rejects_bad_input(b2):
         b2.b2_model_predict_variant(0, 99)
 
 
-def test_sm_predictions(b2):
-    """The model re-targeted at an SM sub-partition: the tensor-core and FP64-FMA kernels are predicted
-    pipe-bound (the model, like the paper's Sandy Bridge table, cannot separate them), the scalar FFMA kernel is
-    predicted issue-bound below the packed-pair kernel -- the order the measurements show."""
+def _predictions(b2):
     pred = {}
     for dtype in (0, 1):
         for v in range(b2.b2_variant_count(dtype)):
             frac, js = b2.b2_model_predict_variant(dtype, v)
             d = json.loads(js)
             assert 0 < frac <= 1 and abs(d["predicted_fraction"] - frac) < 1e-4
+            assert abs(min(d["pipe_fraction"], d["feed_fraction"]) * d["coverage"] * d["stall"] - frac) < 1e-3
             pred[d["variant"]] = (frac, d)
-    f64 = {k: v for k, v in pred.items() if k.startswith("d")}
-    assert all(abs(v[0] - 1.0) < 1e-9 for v in f64.values())
-    for name, (frac, d) in f64.items():
+    return pred
+
+
+def test_sm_predictions(b2):
+    """The model re-targeted at an SM sub-partition, factor by factor.  Pipelines: the tensor-core kernels are bound
+    by the FP64 tensor pipe, the scalar FFMA kernel by issue slots, the packed-pair kernel by the FP32 pipe, on which
+    the moves that duplicate b are jobs too (16 of 80 for the 8 x 8 block, the share the profiler shows).  Stall
+    term: only kernels with a CTA-wide barrier per slab carry it, and more resident CTAs cover more of it.  Coverage
+    grows with the independent tensor instructions per scheduler."""
+    pred = _predictions(b2)
+    for name, (frac, d) in pred.items():
         bound = max(d["clocks_per_k"], key=d["clocks_per_k"].get)
-        assert bound == ("tensor64" if name.startswith("dmma") else "fp64")
-    assert abs(pred["dmma_tma_64x64x16_s3"][1]["measured_fraction"] - 0.97) < 1e-9
-    ffma = pred["ffma_128x64x16_s4"]
-    ffma2 = pred["ffma2_128x64x16_s4"]
-    assert max(ffma[1]["clocks_per_k"], key=ffma[1]["clocks_per_k"].get) == "issue"
-    assert ffma[0] < ffma2[0] and ffma[1]["measured_fraction"] < ffma2[1]["measured_fraction"]
+        if name.startswith("dmma"):
+            assert bound == "tensor64" and d["pipe_fraction"] == 1.0
+        staged_by_tma = "tma" in name or "_ws_" in name
+        assert (d["stall"] == 1.0) == staged_by_tma, name
+    d = pred["ffma2_128x64x16_s4"][1]
+    assert d["jobs_per_k"]["fp32"] == 80.0 and abs(d["pipe_fraction"] - 0.8) < 1e-9
+    assert max(pred["ffma_128x64x16_s4"][1]["clocks_per_k"], key=pred["ffma_128x64x16_s4"][1]["clocks_per_k"].get) == "issue"
     # shared-memory share of the DMMA 64x64 kernel: a quarter of the LSU rate, as the profiler counter shows
     d = pred["dmma_64x64x16_s3"][1]
     assert abs(d["clocks_per_k"]["lsu"] / d["clocks_per_k"]["tensor64"] - 0.25) < 1e-9
+    # W = L + n*k: one CTA on the SM pays the whole barrier stall, two CTAs half of it
+    one, two = pred["dmma_128x128x16_s4"][1], pred["dmma_128x64x16_s3"][1]
+    assert abs(one["stall"] - 2048 / (2048 + 250)) < 1e-3 and abs(two["stall"] - 2048 / (2048 + 125)) < 1e-3
+    assert pred["dmma_tma_32x32x16_s3"][1]["coverage"] < pred["dmma_tma_64x64x16_s3"][1]["coverage"]
+    # Section 5 restated for a thread: N_updates = floor((255 - accumulators - R_A) / R_R) >= 2 for every built kernel,
+    # and the register estimate is close to what the compiler uses (120-128 and 200-218 for the two DMMA warp tiles)
+    assert all(d["n_updates"] >= 2 for _, d in pred.values())
+    assert pred["dmma_64x64x16_s3"][1]["registers"] == 120 and pred["dmma_128x64x16_s3"][1]["registers"] == 200
+    assert abs(pred["dmma_tma_64x64x16_s3"][1]["measured_fraction"] - 0.97) < 1e-9
+
+
+def test_predicted_order_of_built_variants_matches_measured_order(b2):
+    """The paper validates its model by the ORDER it predicts for the candidate kernels against the measured order
+    (Section 6.1, Xeon Phi: preserved but for one mix).  The same check for the variants built here, per data type:
+    no pair whose predicted and measured fractions both differ by more than 0.05 may be ordered the other way round,
+    and every variant the selector may choose is predicted within 0.08 of its measured fraction or is on the
+    short list of known misses (fp32 tiles measured with a k-contiguous B, whose element-wise transposing copy the
+    model does not price)."""
+    pred = _predictions(b2)
+    known_misses = {"ffma2_64x64x16_s4", "ffma2_t4_32x32x16_s4", "ffma2_t16x8_128x128x16_s3"}
+    for prefix in ("d", "f"):
+        items = [(n, f, d["measured_fraction"]) for n, (f, d) in pred.items() if n.startswith(prefix)]
+        for n1, p1, m1 in items:
+            for n2, p2, m2 in items:
+                if n1 in known_misses or n2 in known_misses:
+                    continue
+                if p1 - p2 > 0.05 and m2 - m1 > 0.05:
+                    raise AssertionError(f"{n1} predicted above {n2} ({p1:.3f} > {p2:.3f}) but measured below "
+                                         f"({m1:.3f} < {m2:.3f})")
+        for n, p, m in items:
+            comparison_only = n.startswith(("dfma", "ffma_", "dmma_w8", "dmma_ws"))
+            if n not in known_misses and not comparison_only:
+                assert abs(p - m) <= 0.08, (n, p, m)
+    for n in known_misses:
+        assert pred[n][0] - pred[n][1]["measured_fraction"] > 0.08  # still a miss: take it off the list when fixed
+
+
+def test_enumeration_ranks_candidates_under_the_register_and_shared_memory_limits(b2):
+    """Section 5.1's work flow: every candidate in the list fits the limits, the list is sorted by prediction, every
+    built variant appears with its rank, and the best fp64 candidates are tensor-core kernels fed by the tensor
+    memory accelerator -- the family the library's headline kernel belongs to."""
+    for dtype in (0, 1):
+        e = json.loads(b2.b2_model_enumerate(dtype, 12))
+        ranked = e["ranked"]
+        assert e["candidates"] > 100 and len(ranked) >= 12
+        top = [r for r in ranked if r["rank"] <= 12]
+        assert [r["rank"] for r in top] == list(range(1, 13))
+        assert all(a["predicted_fraction"] >= b["predicted_fraction"] - 1e-9 for a, b in zip(ranked, ranked[1:]))
+        for r in ranked:
+            assert r["registers"] <= 255 and r["n_updates"] >= 2 and r["ctas_per_sm"] >= 1
+            assert r["smem_bytes"] * r["ctas_per_sm"] <= 233472
+            assert r["cta_tile"] == [r["warp_tile"][0] * r["warps"][0], r["warp_tile"][1] * r["warps"][1]]
+        built = {r["built_as"] for r in ranked if r["built_as"]}
+        names = {b2.b2_variant_name(dtype, v) for v in range(b2.b2_variant_count(dtype))}
+        assert built <= names and len(built) >= (5 if dtype == 1 else 8)
+        if dtype == 0:
+            assert all(r["kind"] == "dmma" and r["tma"] for r in top)
+            best_built = min((r for r in ranked if r["built_as"]), key=lambda r: r["rank"])
+            assert "tma" in best_built["built_as"]
+    with pytest.raises(b2.B2Error):
+        b2.b2_model_enumerate(2, 4)
+    with pytest.raises(b2.B2Error):
+        b2.b2_model_enumerate(0, 0)
