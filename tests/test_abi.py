@@ -96,7 +96,7 @@ def test_selector_is_sane_without_gpu(b2):
     for cfg, (m, n) in ((big, (8192, 8192)), (tiny, (256, 256))):
         assert cfg["micro_kernel"].startswith("dmma")
         assert cfg["tiles_m"] * cfg["BM"] >= m and cfg["tiles_n"] * cfg["BN"] >= n
-        assert cfg["grid"] == cfg["tiles_m"] * cfg["tiles_n"]
+        assert cfg["grid"] == cfg["tiles_m"] * cfg["tiles_n"] * cfg["k_split"]
     assert big["micro_kernel"] == "dmma_tma" and tiny["BM"] * tiny["BN"] <= 32 * 32
     f32 = json.loads(b2.b2_gemm_query_config(1, "N", "T", 4096, 4096, 4096, 4096, 4096, 4096))
     assert f32["micro_kernel"] == "ffma2" and f32["dtype"] == "f32"
