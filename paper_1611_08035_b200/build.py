@@ -72,6 +72,15 @@ def build(verbose: bool = False, force: bool = False) -> Path:
     sources = sorted(CSRC.glob("*.cu"))
     if not sources:
         raise RuntimeError("no CUDA sources found")
+    # objects, stamps and logs of sources that no longer exist would be linked / reported: drop them
+    stems = {src.stem for src in sources}
+    stale = False
+    for f in list(BUILD_DIR.iterdir()):
+        stem = f.name.split(".")[0]
+        if f.suffix in (".o", ".stamp", ".log") and stem not in stems:
+            f.unlink()
+            stale = True
+    force = force or stale
     with ThreadPoolExecutor(max_workers=min(8, len(sources))) as ex:
         objs = list(ex.map(lambda s: _compile(s, verbose), sources))
     newest = max(o.stat().st_mtime for o in objs)
