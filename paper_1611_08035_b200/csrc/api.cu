@@ -205,7 +205,8 @@ int choose_variant(int64_t m, int64_t n, int64_t k, bool aligned, int64_t batch 
         TileChoice c = cand[v];
         // reduction: two cluster barriers and, for the first CTA, the other CTAs' accumulators through
         // distributed shared memory
-        c.per_tile_extra_clks += 1500.0 + (split - 1) * (double)vi.bm * vi.bn * sizeof(T) / 32.0 / split;
+        // (about 2000 clocks for the 128 x 64 fp32 tile, where it was fitted; 800 for a 32 x 32 fp64 tile)
+        c.per_tile_extra_clks += 400.0 + (split - 1) * (double)vi.bm * vi.bn * sizeof(T) / 10.0 / split;
         const double t = estimate_clks(c, m, n, k_part, sms, (int)sizeof(T), batch * split);
         if (t < 0.97 * best_t) best = v, best_t = t, *ksplit_out = split;  // a split has to win by 3 %
       }
