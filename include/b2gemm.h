@@ -332,6 +332,21 @@ int b2_sgemm_host(char transa, char transb, int64_t m, int64_t n, int64_t k, flo
 #define B2_PROBE_DMMA_M16N8K8 4
 #define B2_PROBE_DMMA_M16N8K16 5
 #define B2_PROBE_FFMA2 6 /* packed fp32 pair multiply-add, fma.rn.f32x2 */
+/*
+ * Instruction-mix kinds: one round is one 16-deep slab of a GEMM micro-kernel's inner loop -- per k the
+ * shared-memory fragment loads and the multiply-adds of one rank-1 update of the CTA tile, the code the GEMM
+ * kernels run -- over slabs that stay in shared memory (no global traffic, no staging).  threads_per_cta must
+ * be the micro-kernel's CTA size (128, but 64 for the 4 x 4 kind; -2 otherwise); the CTAs per SM are the caller's choice
+ * through `ctas`.  OR-ing B2_PROBE_WITH_BARRIER adds the one CTA-wide barrier per slab of the cp.async-staged
+ * kernels.  The rate such a probe reaches is the ceiling of that instruction mix at that residency.
+ */
+#define B2_PROBE_MIX_FFMA2_8X8 7  /* fp32 128 x 64 tile, 8 x 8 per thread: 32 fma.rn.f32x2 + 4 ld.shared.v4 per k */
+#define B2_PROBE_MIX_FFMA2_16X8 8 /* fp32 128 x 128 tile, 16 x 8 per thread: 64 fma.rn.f32x2 + 6 ld.shared.v4 per k */
+#define B2_PROBE_MIX_DMMA_64X64 9 /* fp64 64 x 64 tile, 32 x 32 per warp: 8 mma.m16n8k4 + 6 fragment loads per 4 k */
+#define B2_PROBE_MIX_FFMA_8X8 10  /* fp32 128 x 64 tile, 8 x 8 per thread, scalar: 64 fma.rn.f32 + 4 ld.shared.v4 per k */
+#define B2_PROBE_MIX_FFMA2_4X4 11 /* fp32 32 x 32 tile of 64 threads, 4 x 4 per thread: 8 fma.rn.f32x2 + 2 ld.shared.v4 */
+#define B2_PROBE_MIX_DFMA_8X8 12  /* fp64 128 x 64 tile, 8 x 8 per thread: 64 fma.rn.f64 + 8 ld.shared.v2 per k */
+#define B2_PROBE_WITH_BARRIER 0x100
 int b2_pipe_probe(int kind, int threads_per_cta, int ctas, int64_t iters, void* scratch, size_t scratch_bytes,
                   double* fma_per_thread_iter, void* cuda_stream);
 

@@ -219,6 +219,18 @@ struct DmmaMicro {
     c = __dadd_rn(c, __longlong_as_double((long long)bits));
   }
 
+  // sum of a lane's accumulators (probes keep their result alive through it)
+  static __device__ __forceinline__ double checksum(const Acc& acc) {
+    double s = 0.0;
+#pragma unroll
+    for (int mi = 0; mi < MI; ++mi)
+#pragma unroll
+      for (int ni = 0; ni < NI; ++ni)
+#pragma unroll
+        for (int r = 0; r < 4; ++r) s += acc.c[mi][ni][r];
+    return s;
+  }
+
   // One BK-deep slab: BK/4 k-steps of MI*NI independent mma.
   static __device__ __forceinline__ void compute(Acc& acc, const double* __restrict__ sA,
                                                  const double* __restrict__ sB, int warp_m, int warp_n, int lane) {
@@ -421,6 +433,16 @@ struct SimtMicro {
     } else {
       return acc.c[i][j];
     }
+  }
+
+  // sum of a thread's accumulators (probes keep their result alive through it)
+  static __device__ __forceinline__ T checksum(const Acc& acc) {
+    T s = T(0);
+#pragma unroll
+    for (int i = 0; i < TM; ++i)
+#pragma unroll
+      for (int j = 0; j < TN; ++j) s += get(acc, i, j);
+    return s;
   }
 
   static __device__ __forceinline__ void load_vec(T* dst, const T* src) {

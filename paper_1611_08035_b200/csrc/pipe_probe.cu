@@ -11,6 +11,7 @@
 #include <stdint.h>
 
 #include "b2gemm.h"
+#include "gemm_kernel.cuh"
 
 namespace {
 
@@ -176,6 +177,83 @@ __global__ void probe_dmma_m16n8k16(long long iters, double* sink, long long* cy
   if (threadIdx.x == 0) cycles[blockIdx.x] = t1 - t0;
 }
 
+// Instruction-mix probes: the inner loop of a GEMM micro-kernel exactly as the GEMM kernels run it (the same
+// compute() the kernels call: per k the shared-memory fragment loads plus the multiply-adds of one rank-1 update)
+// over slabs that sit in shared memory from the start.  No global traffic, no staging code; BARRIER adds the one
+// CTA-wide barrier per slab that the cp.async-staged kernels pass.  What such a probe reaches is the ceiling of the
+// micro-kernel's instruction mix at the given residency; the gap between it and the full kernel is staging.
+constexpr int kMixStages = 2;  // the slab address changes every round, so no load can be hoisted out of the loop
+
+template <class Micro, bool BARRIER>
+__global__ void __launch_bounds__(Micro::NT) probe_mix(long long iters, float* sink, long long* cycles) {
+  using T = typename Micro::T;
+  constexpr int STAGES = kMixStages;
+  extern __shared__ __align__(16) unsigned char mix_smem[];
+  T* sA = reinterpret_cast<T*>(mix_smem);
+  T* sB = sA + STAGES * Micro::A_STAGE;
+  for (int i = threadIdx.x; i < STAGES * Micro::A_STAGE; i += Micro::NT) sA[i] = T(1) + T(1e-3) * T(i % 61);
+  for (int i = threadIdx.x; i < STAGES * Micro::B_STAGE; i += Micro::NT) sB[i] = T(1e-3) * T(1 + i % 53);
+  __syncthreads();
+  constexpr int WARPS_M = Micro::BM / Micro::WTM;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int warp_m = warp % WARPS_M, warp_n = warp / WARPS_M;
+  typename Micro::Acc acc;
+  Micro::zero(acc);
+  long long t0 = clock64();
+  for (long long it = 0; it < iters; ++it) {
+    const int st = (int)(it & (STAGES - 1));
+    Micro::compute(acc, sA + st * Micro::A_STAGE, sB + st * Micro::B_STAGE, warp_m, warp_n, lane);
+    if (BARRIER) __syncthreads();
+  }
+  long long t1 = clock64();
+  const T s = Micro::checksum(acc);
+  if (s == T(-1)) sink[0] = (float)s;
+  if (threadIdx.x == 0) cycles[blockIdx.x] = t1 - t0;
+}
+
+using MixFfma2_8x8 = b2::SimtMicro<float, 128, 64, 16, 2, 2, false, false, true, 8, 8>;
+using MixFfma2_16x8 = b2::SimtMicro<float, 128, 128, 16, 1, 4, false, false, true, 16, 8>;
+using MixDmma_64x64 = b2::DmmaMicro<64, 64, 16, 2, 2, false, false>;
+using MixFfma_8x8 = b2::SimtMicro<float, 128, 64, 16, 2, 2, false, false, false, 8, 8>;
+using MixFfma2_4x4 = b2::SimtMicro<float, 32, 32, 16, 1, 2, false, false, true, 4, 4>;
+using MixDfma_8x8 = b2::SimtMicro<double, 128, 64, 16, 2, 2, false, false, false, 8, 8>;
+
+// Shared memory that nothing touches, behind the slabs, pads each CTA so that exactly ceil(ctas / SMs) of them fit an SM: the
+// probe then runs at the residency the caller asked for, evenly over the SMs, instead of wherever the block
+// scheduler would pack CTAs this small.
+template <class Micro, bool BARRIER>
+int launch_mix_padded(int ctas, long long iters, void* sink, long long* cyc, cudaStream_t st) {
+  int dev = 0, sms = 0, smem_sm = 0, reserved = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return B2_ERR_LAUNCH;
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  cudaDeviceGetAttribute(&smem_sm, cudaDevAttrMaxSharedMemoryPerMultiprocessor, dev);
+  cudaDeviceGetAttribute(&reserved, cudaDevAttrReservedSharedMemoryPerBlock, dev);
+  int optin = 0;
+  cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+  const long long slabs = (long long)kMixStages * (Micro::A_STAGE + Micro::B_STAGE) * sizeof(typename Micro::T);
+  const int per_sm = (ctas + sms - 1) / sms;
+  long long pad = ((long long)smem_sm / per_sm - reserved) / 1024 * 1024;  // slabs first, untouched padding behind
+  if (pad < slabs) pad = slabs;
+  if (pad > optin) pad = optin;
+  if (cudaFuncSetAttribute(probe_mix<Micro, BARRIER>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pad) !=
+      cudaSuccess)
+    return B2_ERR_LAUNCH;
+  // ask for the largest shared-memory carve-out, or the padded CTAs may not all fit beside the L1
+  cudaFuncSetAttribute(probe_mix<Micro, BARRIER>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                       cudaSharedmemCarveoutMaxShared);
+  probe_mix<Micro, BARRIER><<<ctas, Micro::NT, (size_t)pad, st>>>(iters, (float*)sink, cyc);
+  return 0;
+}
+
+template <class Micro>
+int launch_mix(bool barrier, int threads_per_cta, int ctas, long long iters, void* sink, long long* cyc,
+               double* fma_per_thread_iter, cudaStream_t st) {
+  if (threads_per_cta != Micro::NT) return -2;
+  *fma_per_thread_iter = (double)Micro::BM * Micro::BN * Micro::BK / Micro::NT;
+  return barrier ? launch_mix_padded<Micro, true>(ctas, iters, sink, cyc, st)
+                 : launch_mix_padded<Micro, false>(ctas, iters, sink, cyc, st);
+}
+
 }  // namespace
 
 extern "C" int b2_pipe_probe(int kind, int threads_per_cta, int ctas, int64_t iters, void* scratch,
@@ -190,6 +268,7 @@ extern "C" int b2_pipe_probe(int kind, int threads_per_cta, int ctas, int64_t it
   double* sink = (double*)scratch;
   long long* cyc = (long long*)((char*)scratch + 64);
   constexpr int NS = 8;
+  const bool barrier = (kind & B2_PROBE_WITH_BARRIER) != 0;
   switch (kind) {
     case B2_PROBE_DFMA:
       probe_dfma<<<ctas, threads_per_cta, 0, st>>>(iters, sink, cyc);
@@ -218,6 +297,36 @@ extern "C" int b2_pipe_probe(int kind, int threads_per_cta, int ctas, int64_t it
     case B2_PROBE_DMMA_M16N8K16:
       probe_dmma_m16n8k16<NS><<<ctas, threads_per_cta, 0, st>>>(iters, sink, cyc);
       *fma_per_thread_iter = NS * 16.0 * 8 * 16 / 32;
+      break;
+    case B2_PROBE_MIX_FFMA2_8X8:
+    case B2_PROBE_MIX_FFMA2_8X8 | B2_PROBE_WITH_BARRIER:
+      if (int rc = launch_mix<MixFfma2_8x8>(barrier, threads_per_cta, ctas, iters, sink, cyc, fma_per_thread_iter, st))
+        return rc;
+      break;
+    case B2_PROBE_MIX_FFMA2_16X8:
+    case B2_PROBE_MIX_FFMA2_16X8 | B2_PROBE_WITH_BARRIER:
+      if (int rc = launch_mix<MixFfma2_16x8>(barrier, threads_per_cta, ctas, iters, sink, cyc, fma_per_thread_iter, st))
+        return rc;
+      break;
+    case B2_PROBE_MIX_DMMA_64X64:
+    case B2_PROBE_MIX_DMMA_64X64 | B2_PROBE_WITH_BARRIER:
+      if (int rc = launch_mix<MixDmma_64x64>(barrier, threads_per_cta, ctas, iters, sink, cyc, fma_per_thread_iter, st))
+        return rc;
+      break;
+    case B2_PROBE_MIX_FFMA_8X8:
+    case B2_PROBE_MIX_FFMA_8X8 | B2_PROBE_WITH_BARRIER:
+      if (int rc = launch_mix<MixFfma_8x8>(barrier, threads_per_cta, ctas, iters, sink, cyc, fma_per_thread_iter, st))
+        return rc;
+      break;
+    case B2_PROBE_MIX_FFMA2_4X4:
+    case B2_PROBE_MIX_FFMA2_4X4 | B2_PROBE_WITH_BARRIER:
+      if (int rc = launch_mix<MixFfma2_4x4>(barrier, threads_per_cta, ctas, iters, sink, cyc, fma_per_thread_iter, st))
+        return rc;
+      break;
+    case B2_PROBE_MIX_DFMA_8X8:
+    case B2_PROBE_MIX_DFMA_8X8 | B2_PROBE_WITH_BARRIER:
+      if (int rc = launch_mix<MixDfma_8x8>(barrier, threads_per_cta, ctas, iters, sink, cyc, fma_per_thread_iter, st))
+        return rc;
       break;
     default:
       return -1;

@@ -82,7 +82,10 @@ inline WarpMix warp_mix(int kind, int wtm, int wtn, int staging_per_slab, int sl
   WarpMix m;
   for (int i = 0; i < NPIPES; ++i) m.jobs[i] = 0.0;
   m.fma_per_k = (double)wtm * wtn;
-  const double overhead = (staging_per_slab * 3.0 + 12.0) / slab_k;  // staging, barrier, loop control per k
+  // staging (copy instruction plus its 64-bit address arithmetic), barrier, loop control per k: the profiler counts
+  // 5.5 instructions per k beside the multiply-adds and fragment loads in the fp32 128 x 64 kernel, 7 to 8 in the
+  // 128 x 128 one
+  const double overhead = (staging_per_slab * 6.0 + 24.0) / slab_k;
   if (kind == MK_DMMA) {
     const double mi = wtm / 16.0, ni = wtn / 8.0;
     m.jobs[TENSOR64] = mi * ni / 4.0;           // one mma covers four k
@@ -102,11 +105,15 @@ inline WarpMix warp_mix(int kind, int wtm, int wtn, int staging_per_slab, int sl
       m.jobs[FP32] = fma;
       m.jobs[ISSUE] = fma * kScalarFmaSlots + loads + overhead;
     } else {
-      // 32 packed instructions, two jobs each, plus the moves that copy each of the tn values of b into both halves
-      // of a pair: two 32-bit moves per value, executed on the same FP32 pipe (the profiler puts them at a fifth of
-      // that pipe's activity in the 8 x 8 kernel: 16 of 80 jobs)
-      m.jobs[FP32] = fma + 2.0 * tn;
-      m.jobs[ISSUE] = fma / 2.0 + loads + 2.0 * tn + overhead;
+      // A packed pair instruction is two jobs on the FP32 pipe and holds the sub-partition's dispatch port for two
+      // clocks (it reads three 64-bit operands per lane); so does a 16-byte shared-memory load.  At peak the pair
+      // instructions alone fill the port, and every other instruction takes its slots from them: the loop of an
+      // 8 x 8 block needs 64 + 8 slots per rank-1 update, of a 16 x 8 block 128 + 12.  The instruction-mix probes
+      // (the inner loops over resident slabs, nothing else) measure 0.87 and 0.92 of the pipe's peak; the raw
+      // pair instruction reaches 0.97.  (Copying a value of b into both halves of a pair costs nothing: the
+      // profiler counts no instruction for it.)
+      m.jobs[FP32] = fma;
+      m.jobs[ISSUE] = fma + 2.0 * loads + overhead;
     }
   }
   return m;

@@ -22,11 +22,24 @@ KINDS = {
     "dmma_m16n8k8": 4,
     "dmma_m16n8k16": 5,
     "ffma2": 6,
+    "mix_ffma2_8x8": 7,
+    "mix_ffma2_16x8": 8,
+    "mix_dmma_64x64": 9,
+    "mix_ffma_8x8": 10,
+    "mix_ffma2_4x4": 11,
+    "mix_dfma_8x8": 12,
 }
+WITH_BARRIER = 0x100  # OR-ed into a mix kind: one CTA-wide barrier per slab
+# residencies at which the GEMM kernels run each mix (CTAs of 128 threads per SM), plus one above and below
+MIX_RESIDENCY = {"mix_ffma2_8x8": (2, 3, 4), "mix_ffma2_16x8": (1, 2), "mix_dmma_64x64": (2, 3, 4),
+                 "mix_ffma_8x8": (3, 4), "mix_ffma2_4x4": (4, 8), "mix_dfma_8x8": (1, 2)}
+MIX_THREADS = {"mix_ffma2_4x4": 64}
 
 
-def probe(kind: str, threads_per_cta: int, ctas_per_sm: int, iters: int, repeats: int = 3) -> dict:
+def probe(kind: str, threads_per_cta: int, ctas_per_sm: int, iters: int, repeats: int = 3,
+          barrier: bool = False) -> dict:
     lib = binding.lib()
+    code = KINDS[kind] | (WITH_BARRIER if barrier else 0)
     dev = torch.device("cuda", torch.cuda.current_device())
     sms = torch.cuda.get_device_properties(dev).multi_processor_count
     ctas = sms * ctas_per_sm
@@ -37,7 +50,7 @@ def probe(kind: str, threads_per_cta: int, ctas_per_sm: int, iters: int, repeats
     for _ in range(repeats):
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
-        rc = lib.b2_pipe_probe(KINDS[kind], threads_per_cta, ctas, iters, scratch.data_ptr(), scratch.numel(),
+        rc = lib.b2_pipe_probe(code, threads_per_cta, ctas, iters, scratch.data_ptr(), scratch.numel(),
                                ctypes.byref(per), stream)
         e1.record()
         if rc != 0:
@@ -46,10 +59,12 @@ def probe(kind: str, threads_per_cta: int, ctas_per_sm: int, iters: int, repeats
         ms = e0.elapsed_time(e1)
         if best_ms is None or ms < best_ms:
             best_ms = ms
-            cycles = scratch[64:].view(torch.int64).double().mean().item()
+            # the slowest CTA: CTAs that share an SM do not get equal shares of it, so the early finishers'
+            # cycle counts understate the time the work took
+            cycles = scratch[64:].view(torch.int64).double().max().item()
     fma_total = float(threads_per_cta) * ctas * iters * per.value
     return {
-        "kind": kind,
+        "kind": kind + ("+barrier" if barrier else ""),
         "threads_per_cta": threads_per_cta,
         "ctas_per_sm": ctas_per_sm,
         "iters": iters,
@@ -66,6 +81,11 @@ def main() -> None:
     ap.add_argument("--long-iters", type=int, default=0, help="also run each kind this long (sustained clocks)")
     args = ap.parse_args()
     for kind in KINDS:
+        if kind in MIX_RESIDENCY:
+            for cps in MIX_RESIDENCY[kind]:
+                for barrier in (False, True):
+                    print(json.dumps(probe(kind, MIX_THREADS.get(kind, 128), cps, max(1, args.iters // 16), barrier=barrier)), flush=True)
+            continue
         for tpc, cps in ((128, 1), (256, 1), (128, 2), (256, 2), (512, 2)):
             print(json.dumps(probe(kind, tpc, cps, args.iters)), flush=True)
         if args.long_iters:

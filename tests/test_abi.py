@@ -68,6 +68,9 @@ def test_argument_checks_need_no_gpu(b2):
     assert lib.b2_pipe_probe(99, 128, 1, 10, fake, 4096, ctypes.byref(per), None) == -1
     assert lib.b2_pipe_probe(0, 100, 1, 10, fake, 4096, ctypes.byref(per), None) == -2
     assert lib.b2_pipe_probe(0, 128, 1, 10, fake, 8, ctypes.byref(per), None) == -6
+    # instruction-mix kinds run a micro-kernel's inner loop and take that micro-kernel's CTA size only
+    assert lib.b2_pipe_probe(7, 256, 1, 10, fake, 4096, ctypes.byref(per), None) == -2
+    assert lib.b2_pipe_probe(11 | 0x100, 128, 1, 10, fake, 4096, ctypes.byref(per), None) == -2
 
 
 def test_workspace_sizes(b2):

@@ -402,6 +402,21 @@ def test_pipe_probe_rates(b2):
     assert 110 <= f["fma_per_clk_per_sm"] <= 132
 
 
+def test_instruction_mix_probes(b2):
+    """The inner loops of the micro-kernels over resident slabs: the tensor-core mix runs at the pipe's rate, the
+    packed-pair mixes below theirs (the shared-memory loads take issue slots from the pair instructions) and in
+    the order of their loads per multiply-add: 16 x 8 above 8 x 8 above 4 x 4; the barrier costs a few percent."""
+    from paper_1611_08035_b200 import pipes
+    rate = lambda kind, cps, thr=128, **kw: pipes.probe(kind, thr, cps, 2000, **kw)["tflops"]
+    dm = rate("mix_dmma_64x64", 2)
+    f8, f8b = rate("mix_ffma2_8x8", 3), rate("mix_ffma2_8x8", 3, barrier=True)
+    f16 = rate("mix_ffma2_16x8", 2)
+    f4 = rate("mix_ffma2_4x4", 8, thr=64)
+    assert 0.93 * 37.2 <= dm <= 1.02 * 37.2
+    assert 0.78 * 74.4 <= f8 <= 0.95 * 74.4 and 0.93 * f8 <= f8b <= 1.01 * f8
+    assert f4 < f8 < f16 <= 0.99 * 74.4
+
+
 @pytest.mark.parametrize("kind", ["d", "s"])
 def test_more_than_2_31_elements_of_c(b2, oracle, kind):
     """C with more than 2^31 elements (46400^2): column offsets no longer fit 32 bits even in elements.  k is short,

@@ -134,8 +134,10 @@ def _predictions(b2):
 
 def test_sm_predictions(b2):
     """The model re-targeted at an SM sub-partition, factor by factor.  Pipelines: the tensor-core kernels are bound
-    by the FP64 tensor pipe, the scalar FFMA kernel by issue slots, the packed-pair kernel by the FP32 pipe, on which
-    the moves that duplicate b are jobs too (16 of 80 for the 8 x 8 block, the share the profiler shows).  Stall
+    by the FP64 tensor pipe, the scalar FFMA kernel and the packed-pair kernels by issue slots: a pair instruction and a
+    16-byte shared-memory load hold the dispatch port for two clocks each, so the 8 x 8 block's 64 + 8 slots per
+    rank-1 update leave 0.87 of the FP32 pipe at best and the 16 x 8 block's 128 + 12 leave 0.91, which is what the
+    instruction-mix probes measure (0.87, 0.92).  Stall
     term: only kernels with a CTA-wide barrier per slab carry it, and more resident CTAs cover more of it.  Coverage
     grows with the independent tensor instructions per scheduler."""
     pred = _predictions(b2)
@@ -146,7 +148,10 @@ def test_sm_predictions(b2):
         staged_by_tma = "tma" in name or "_ws_" in name
         assert (d["stall"] == 1.0) == staged_by_tma, name
     d = pred["ffma2_128x64x16_s4"][1]
-    assert d["jobs_per_k"]["fp32"] == 80.0 and abs(d["pipe_fraction"] - 0.8) < 1e-9
+    assert d["jobs_per_k"]["fp32"] == 64.0 and max(d["clocks_per_k"], key=d["clocks_per_k"].get) == "issue"
+    assert 64 / (72 + 4) < d["pipe_fraction"] < 64 / 72  # slots of the loop itself, plus a few for staging
+    wide = pred["ffma2_t16x8_128x128x16_s3"][1]
+    assert 128 / (140 + 5) < wide["pipe_fraction"] < 128 / 140 and wide["pipe_fraction"] > d["pipe_fraction"]
     assert max(pred["ffma_128x64x16_s4"][1]["clocks_per_k"], key=pred["ffma_128x64x16_s4"][1]["clocks_per_k"].get) == "issue"
     # shared-memory share of the DMMA 64x64 kernel: a quarter of the LSU rate, as the profiler counter shows
     d = pred["dmma_64x64x16_s3"][1]
