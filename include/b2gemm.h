@@ -79,7 +79,10 @@ int b2_sgemm(char transa, char transb, int64_t m, int64_t n, int64_t k, float al
 /*
  * The same two operations with an explicit kernel variant, 0 <= variant < b2_variant_count(dtype),
  * or B2_VARIANT_AUTO.  Used by tests and benchmarks to exercise every micro-kernel; a variant
- * that cannot serve the given shape/alignment returns B2_ERR_VARIANT and launches nothing.
+ * that cannot serve the given shape/alignment returns B2_ERR_VARIANT and launches nothing
+ * (the TMA-staged variants need 16-byte aligned columns of A and B; the fp32 one, "ffma2_tma",
+ * reads each operand in the layout it has in memory and also declines transa = T with transb = N,
+ * where neither operand has its C index contiguous).
  * An explicit variant is launched with one CTA per tile; variant + 256*s (s = 2 or 4) asks for
  * the k-loop of every tile to be split over a thread-block cluster of s CTAs, whose partial
  * sums are added in rank order through distributed shared memory (Section 2's kc loop, cut in

@@ -31,6 +31,7 @@ int launch_f32_v1(const GemmArgs<float>&, bool, bool, bool, cudaStream_t);
 int launch_f32_v2(const GemmArgs<float>&, bool, bool, bool, cudaStream_t);
 int launch_f32_v3(const GemmArgs<float>&, bool, bool, bool, cudaStream_t);
 int launch_f32_s32(const GemmArgs<float>&, bool, bool, bool, cudaStream_t);
+int launch_f32_tma(const GemmArgs<float>&, bool, bool, bool, cudaStream_t);
 
 model::SmPrediction predict_variant(int dtype, int variant);  // model_api.cu
 
@@ -63,8 +64,10 @@ const VariantInfo kF32Info[] = {
     {"ffma2_64x64x16_s4", "ffma2", 64, 64, 16, 4, 64, 6, 0.64},
     {"ffma_128x64x16_s4", "ffma", 128, 64, 16, 4, 128, 4, 0.70},
     {"ffma2_t4_32x32x16_s4", "ffma2", 32, 32, 16, 4, 64, 8, 0.40, 4, 4, 0.0, 7.0, true},
+    {"ffma2_tma_128x128x16_s6", "ffma2_tma", 128, 128, 16, 6, 128, 2, 0.785, 16, 8},
 };
-const LaunchFn<float> kF32Launch[] = {launch_f32_v0, launch_f32_v1, launch_f32_v2, launch_f32_v3, launch_f32_s32};
+const LaunchFn<float> kF32Launch[] = {launch_f32_v0, launch_f32_v1, launch_f32_v2,
+                                      launch_f32_v3, launch_f32_s32, launch_f32_tma};
 
 }  // namespace
 
@@ -155,8 +158,9 @@ int choose_variant(int64_t m, int64_t n, int64_t k, bool aligned, int64_t batch 
     // measured counterparts, never chosen automatically: the FMA micro-kernels on fp64 / scalar fp32, the
     // eight-warp 64 x 64 tile (slower than the four-warp one wherever it was measured) and the persistent kernel
     const bool comparison_only = strcmp(vi.micro, "dfma") == 0 || strcmp(vi.micro, "ffma") == 0 ||
-                                 strcmp(vi.micro, "dmma_ws") == 0 || strcmp(vi.micro, "dmma_w8") == 0;
-    const bool needs_alignment = strcmp(vi.micro, "dmma_tma") == 0;
+                                 strcmp(vi.micro, "dmma_ws") == 0 || strcmp(vi.micro, "dmma_w8") == 0 ||
+                                 strcmp(vi.micro, "ffma2_tma") == 0;
+    const bool needs_alignment = strcmp(vi.micro, "dmma_tma") == 0 || strcmp(vi.micro, "ffma2_tma") == 0;
     // Steady-state fraction of the arithmetic pipe at full residency: the pipeline model's prediction (Section 4
     // estimate x latency coverage x barrier stall, queue_model.h).  The table's measured value is the recorded check
     // of that prediction; it replaces it only where the two are more than kModelTrust apart (fp32 tiles whose

@@ -113,27 +113,40 @@ __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wa
 // 2-D fp64 tensor map of a column-major matrix (rows contiguous, leading dimension ld) with the given box.
 bool make_map(CUtensorMap* map, const double* base, int64_t rows, int64_t cols, int64_t ld, int box_inner,
               int box_outer);
+// The same for fp32; swizzle64: the 16-byte pieces of every 64-byte box row are permuted (piece index XOR bits
+// 7-8 of the shared-memory address), so that pieces of consecutive rows fall into different banks.
+bool make_map_f32(CUtensorMap* map, const float* base, int64_t rows, int64_t cols, int64_t ld, int box_inner,
+                  int box_outer, bool swizzle64);
 // Device address (on the current device) of the status word that bounded waits write; nullptr on failure.
 int* status_pointer();
 
 // ---- the kernel ------------------------------------------------------------------------------
-template <class Micro, int STAGES, bool TA, bool TB>
+// LAG: the producer refills, before it multiplies slab kt, the slot of slab kt - LAG, so STAGES - LAG slabs are in
+// flight or ready.  With LAG = 1 the producing thread waits at every slab until the slowest warp of the CTA has
+// released the slab just finished, and its own warp with it; LAG = 2 asks for a slot that all warps left a whole
+// slab ago.
+template <class Micro, int STAGES, bool TA, bool TB, int LAG = 1>
 struct GemmTmaKernel {
-  using T = double;
-  static_assert(std::is_same<typename Micro::T, double>::value, "TMA staging is instantiated for the fp64 DMMA kernels");
+  static_assert(LAG >= 1 && LAG < STAGES, "at least one slab must be in flight");
+  using T = typename Micro::T;
   static constexpr int BM = Micro::BM, BN = Micro::BN, BK = Micro::BK, NT = Micro::NT;
   static constexpr int NWARPS = NT / 32;
   // boxes: inner extent = shared-memory pitch, outer extent = number of lines of the staged tile
   static constexpr int A_INNER = Micro::PA, A_OUTER = TA ? BM : BK;
   static constexpr int B_INNER = Micro::PB, B_OUTER = TB ? BK : BN;
   static_assert(A_INNER * A_OUTER == Micro::A_STAGE && B_INNER * B_OUTER == Micro::B_STAGE, "boxes tile the stages");
-  static constexpr uint32_t A_BYTES = Micro::A_STAGE * 8, B_BYTES = Micro::B_STAGE * 8;
-  static_assert(A_BYTES % 128 == 0 && B_BYTES % 128 == 0, "stages must keep 128-byte alignment");
-  static constexpr size_t SMEM_BYTES = (size_t)STAGES * (A_BYTES + B_BYTES) + 2 * STAGES * sizeof(uint64_t);
+  static constexpr uint32_t A_BYTES = Micro::A_STAGE * sizeof(T), B_BYTES = Micro::B_STAGE * sizeof(T);
+  // swizzled boxes (fp32, k-contiguous operands) repeat their pattern every 512 bytes: stages start on 1024
+  static constexpr uint32_t ALIGN = sizeof(T) == 4 ? 1024 : 128;
+  static_assert(A_BYTES % ALIGN == 0 && B_BYTES % ALIGN == 0, "stages must keep their alignment");
+  static constexpr size_t SMEM_BYTES =
+      (size_t)STAGES * (A_BYTES + B_BYTES) + 2 * STAGES * sizeof(uint64_t) + (ALIGN > 128 ? ALIGN : 0);
 
   static __device__ __forceinline__ void run(const GemmArgs<T>& p, const CUtensorMap* mapA, const CUtensorMap* mapB,
                                              int* status) {
-    extern __shared__ __align__(128) unsigned char smem_raw[];
+    extern __shared__ __align__(128) unsigned char smem_dyn[];
+    unsigned char* smem_raw = smem_dyn;
+    if constexpr (ALIGN > 128) smem_raw += (ALIGN - (smem_u32(smem_dyn) & (ALIGN - 1))) & (ALIGN - 1);
     T* sA = reinterpret_cast<T*>(smem_raw);
     T* sB = sA + STAGES * Micro::A_STAGE;
     uint64_t* full = reinterpret_cast<uint64_t*>(smem_raw + (size_t)STAGES * (A_BYTES + B_BYTES));
@@ -169,7 +182,7 @@ struct GemmTmaKernel {
 
     int issued = 0;  // slabs handed to the TMA so far (thread 0 only)
     if (tid == 0) {
-      for (; issued < STAGES - 1 && issued < KT; ++issued) issue(issued);
+      for (; issued < STAGES - LAG && issued < KT; ++issued) issue(issued);
     }
 
     // beta != 0: pull the tile's old C values towards L2 while the k-loop runs
@@ -192,7 +205,7 @@ struct GemmTmaKernel {
     int waited = 0;  // slabs whose arrival this thread has seen
     for (int kt = 0; kt < KT; ++kt) {
       const int slot = kt % STAGES;
-      // refill the slot that slab kt-1 used, once every warp has released it
+      // refill the slot that slab kt - LAG used, once every warp has released it
       if (tid == 0 && issued < KT) {
         const int fslot = issued % STAGES;
         const int round = issued / STAGES;  // how many times this slot has been filled before
@@ -240,7 +253,7 @@ struct GemmTmaKernel {
 
 template <class Kernel, int MIN_CTAS>
 __global__ void __launch_bounds__(Kernel::NT, MIN_CTAS)
-    gemm_tma_kernel(const GemmArgs<double> p, const __grid_constant__ CUtensorMap mapA,
+    gemm_tma_kernel(const GemmArgs<typename Kernel::T> p, const __grid_constant__ CUtensorMap mapA,
                     const __grid_constant__ CUtensorMap mapB, int* status) {
   Kernel::run(p, &mapA, &mapB, status);
 }

@@ -46,7 +46,7 @@ namespace {
 int kind_of(const VariantInfo& vi) {
   if (strncmp(vi.micro, "dmma", 4) == 0) return model::MK_DMMA;
   if (strcmp(vi.micro, "dfma") == 0) return model::MK_DFMA;
-  if (strcmp(vi.micro, "ffma2") == 0) return model::MK_FFMA2;
+  if (strncmp(vi.micro, "ffma2", 5) == 0) return model::MK_FFMA2;
   return model::MK_FFMA;
 }
 }  // namespace
@@ -65,7 +65,7 @@ model::SmCandidate candidate_of(const VariantInfo& vi) {
     c.warps_m = vi.bm / c.wtm, c.warps_n = vi.bn / c.wtn;
   }
   c.bk = vi.bk, c.stages = vi.stages;
-  c.tma = strcmp(vi.micro, "dmma_tma") == 0 || strcmp(vi.micro, "dmma_ws") == 0;
+  c.tma = strcmp(vi.micro, "dmma_tma") == 0 || strcmp(vi.micro, "dmma_ws") == 0 || strcmp(vi.micro, "ffma2_tma") == 0;
   return c;
 }
 
@@ -91,7 +91,7 @@ extern "C" int b2_model_predict_variant(int dtype, int variant, double* fraction
   const int elem = dtype == B2_F64 ? 8 : 4;
   const int threads = 32 * c.warps_m * c.warps_n;
   const int staging = (vi.bm + vi.bn) * vi.bk * elem / 16 / threads;  // 16-byte chunks per thread per slab
-  const WarpMix mix = warp_mix(c.kind, c.wtm, c.wtn, staging > 0 ? staging : 1, vi.bk);
+  const WarpMix mix = warp_mix(c.kind, c.wtm, c.wtn, c.tma ? 0 : (staging > 0 ? staging : 1), vi.bk);
   *fraction = pr.fraction;
   if (json_out) {
     double rate[NPIPES];

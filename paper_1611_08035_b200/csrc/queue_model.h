@@ -219,7 +219,8 @@ inline SmPrediction predict(const SmCandidate& c, const SmLimits& lim, int elem_
   r.feasible = r.n_updates >= 2 && ctas >= 1 && r.regs_per_thread <= lim.max_regs_per_thread && c.wtm > 0 && c.wtn > 0;
   if (!r.feasible) return r;
   const int staging = (r.bm + r.bn) * c.bk * elem_bytes / 16 / r.threads;
-  const WarpMix mix = warp_mix(c.kind, c.wtm, c.wtn, staging > 0 ? staging : 1, c.bk);
+  // slabs that the tensor memory accelerator brings cost the multiplying warps no copy instructions
+  const WarpMix mix = warp_mix(c.kind, c.wtm, c.wtn, c.tma ? 0 : (staging > 0 ? staging : 1), c.bk);
   r.pipe_fraction = predicted_fraction(mix, elem_bytes == 8);
   const double fma_per_clk = elem_bytes == 8 ? 64.0 : 128.0;
   const double bytes_per_fma = (double)(r.bm + r.bn) * elem_bytes / ((double)r.bm * r.bn);

@@ -10,7 +10,7 @@ import numpy as np
 import pytest
 import torch
 
-from gpu_util import run_and_check, sample_columns, staged_by_tma
+from gpu_util import declines_transposes, run_and_check, sample_columns, staged_by_tma
 from paper_1611_08035_b200 import synth
 
 pytestmark = pytest.mark.gpu
@@ -134,20 +134,25 @@ def test_all_variants_multi_tile_ragged(b2, oracle, kind):
                           expect_exact=True)
 
 
-def test_tma_variants_aligned_ragged_shapes(b2, oracle):
+@pytest.mark.parametrize("kind", ["d", "s"])
+def test_tma_variants_aligned_ragged_shapes(b2, oracle, kind):
     """The TMA-staged variants on shapes with ragged m, n and k (edge tiles and the partial last slab are
-    zero-filled by the hardware), even leading dimensions for A and B, an odd one for C."""
-    tma = [v for v in range(nvariants(b2, "d")) if staged_by_tma(b2.b2_variant_name(0, v))]
-    assert len(tma) >= 3
+    zero-filled by the hardware), leading dimensions of A and B that are whole 16-byte units, an odd one for C.
+    fp32: the boxes of k-contiguous operands are swizzled, and each transpose pair runs its own inner loop."""
+    dt = 0 if kind == "d" else 1
+    vec = 2 if kind == "d" else 4
+    tma = [v for v in range(nvariants(b2, kind)) if staged_by_tma(b2.b2_variant_name(dt, v))]
+    assert len(tma) >= (3 if kind == "d" else 1)
     for v in tma:
         for ta, tb in TRANS:
+            if declines_transposes(b2.b2_variant_name(dt, v), ta, tb):
+                continue
             for (m, n, k) in [(200, 136, 75), (129, 65, 17), (1, 1, 1), (7, 300, 33), (333, 270, 145), (64, 64, 1030)]:
                 (ra, _), (rb, _) = synth.operand_shapes(ta, tb, m, n, k)
-                lds = ((ra + 1) // 2 * 2 + 2, (rb + 1) // 2 * 2, m + (m + 1) % 2 + 0)
-                lds = (lds[0], lds[1], m | 1)
-                r = run_and_check(b2, oracle, "d", ta, tb, m, n, k, 0.7, -0.3, seed=m + k, variant=v, lds=lds)
+                lds = ((ra + vec - 1) // vec * vec + vec, (rb + vec - 1) // vec * vec, m | 1)
+                r = run_and_check(b2, oracle, kind, ta, tb, m, n, k, 0.7, -0.3, seed=m + k, variant=v, lds=lds)
                 assert r is not None
-                r = run_and_check(b2, oracle, "d", ta, tb, m, n, k, 1.5, 0.5, dist="int9", seed=m + k, variant=v,
+                r = run_and_check(b2, oracle, kind, ta, tb, m, n, k, 1.5, 0.5, dist="int9", seed=m + k, variant=v,
                                   lds=lds, expect_exact=True)
                 assert r is not None
 

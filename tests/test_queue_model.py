@@ -186,7 +186,7 @@ def test_predicted_order_of_built_variants_matches_measured_order(b2):
                     raise AssertionError(f"{n1} predicted above {n2} ({p1:.3f} > {p2:.3f}) but measured below "
                                          f"({m1:.3f} < {m2:.3f})")
         for n, p, m in items:
-            comparison_only = n.startswith(("dfma", "ffma_", "dmma_w8", "dmma_ws"))
+            comparison_only = n.startswith(("dfma", "ffma_", "dmma_w8", "dmma_ws", "ffma2_tma"))
             if n not in known_misses and not comparison_only:
                 assert abs(p - m) <= 0.08, (n, p, m)
     for n in known_misses:

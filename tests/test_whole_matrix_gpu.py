@@ -14,7 +14,7 @@ import numpy as np
 import pytest
 import torch
 
-from gpu_util import sample_columns, staged_by_tma
+from gpu_util import declines_transposes, sample_columns, staged_by_tma
 from paper_1611_08035_b200 import synth
 
 pytestmark = pytest.mark.gpu
@@ -91,6 +91,8 @@ def test_fp32_cluster_k_split_against_unsplit_2048(b2, oracle):
             auto = C.clone()
             b2.b2_sgemm(ta, tb, m, n, k, 1.5, A, lda, B, ldb, 0.5, auto, ldc)
             for v in range(b2.b2_variant_count(1)):
+                if declines_transposes(b2.b2_variant_name(1, v), ta, tb):
+                    continue
                 Cd = C.clone()
                 b2.b2_sgemm(ta, tb, m, n, k, 1.5, A, lda, B, ldb, 0.5, Cd, ldc, variant=v)
                 _assert_same(Cd, auto, f"{b2.b2_variant_name(1, v)} {ta}{tb} against the automatic (k_split "
