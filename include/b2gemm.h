@@ -304,10 +304,16 @@ int b2_sgemm_tf32x3(char transa, char transb, int64_t m, int64_t n, int64_t k, f
  * Host-buffer forms: A, B, C are HOST pointers (pinned memory makes the copies asynchronous),
  * dev_workspace is DEVICE memory of at least b2_gemm_host_workspace_bytes(...) bytes owned by
  * the caller.  The call copies the referenced parts of A and B (and C when beta != 0) to the
- * device, runs the same kernel as b2_dgemm / b2_sgemm, copies the m x n result back into C and
- * synchronises the stream before returning.  Copies and compute are pipelined over column panels of
- * C on two helper streams that the library creates on its first such call on a device and keeps
- * (no device memory is allocated); these calls are serialised among host threads.
+ * device, runs the kernels of b2_dgemm / b2_sgemm, copies the m x n result back into C and
+ * synchronises the stream before returning.  Copies and compute are pipelined on two helper streams
+ * that the library creates on its first such call on a device and keeps (no device memory is
+ * allocated); these calls are serialised among host threads.  Problems with k < 2048 or fewer than
+ * 2^22 elements of C are pipelined over column panels of C, each panel one b2_dgemm / b2_sgemm
+ * call: the same bits as the device form.  Larger ones travel and are multiplied chunk by chunk
+ * along k, so that the multiplication starts when an eighth of A and B has arrived, and finish
+ * column panel by column panel, so that the copy back overlaps it: C = (...((alpha A_1 B_1) +
+ * alpha A_2 B_2) + ...) + beta C, the same error bound as the single call, exact on integer
+ * data, not the same rounding otherwise; their workspace holds a second buffer of C's size.
  * Argument numbering as b2_dgemm, workspace = 14.
  */
 size_t b2_gemm_host_workspace_bytes(int dtype, char transa, char transb, int64_t m, int64_t n, int64_t k);

@@ -1,11 +1,21 @@
 // Host-buffer forms of the real GEMM: copy the referenced parts of A, B (and C when beta != 0)
 // into the caller's device workspace, run the device entry point, copy the result back.
 //
-// The copies and the multiplication are pipelined over column panels of C: A goes up first, then the panels
-// of B (and of C when beta != 0) follow on a copy-in stream while the kernel works on the panels that have
-// arrived and a copy-out stream returns finished panels -- PCIe is full duplex, so the call takes about
-// max(copy time, compute time) instead of their sum.  The two helper streams and a few events are created on
-// the first call on a device and kept (no device memory is allocated); calls are serialised by a mutex.
+// Copies and multiplication are pipelined on a copy-in stream, the caller's stream and a copy-out stream (PCIe is
+// full duplex), in one of two orders:
+//   * column panels of C (small and medium problems): A goes up first, then the panels of B (and of C when
+//     beta != 0) follow while the kernel works on the panels that have arrived and finished panels go back.
+//     Each panel is one call of the device entry point: the same bits as b2_dgemm / b2_sgemm.  The time is the
+//     upload of A plus about max(copy time, compute time).
+//   * k-chunks first (large problems, k >= 2048): A's upload alone would leave the GPU idle for as long as a
+//     third of the multiplication takes, so A and B go up chunk by chunk along k and the kernel adds
+//     alpha * A_p * B_p to all of C as each chunk p arrives (beta = 0 for the first chunk, 1 afterwards); C's old
+//     values travel last, into a buffer of their own; the last chunk runs column panel by column panel, each
+//     followed by C_panel += beta * C_old_panel and its copy back.  Only the first chunk's upload and the last
+//     panel's download are exposed.  The sum over k is formed chunk by chunk: the same error bound as the single
+//     call, not the same rounding.
+// The two helper streams and a few events are created on the first call on a device and kept (no device memory is
+// allocated); calls are serialised by a mutex.
 #include <mutex>
 
 #include "b2gemm.h"
@@ -16,8 +26,13 @@ namespace {
 
 struct HostPlan {
   int64_t ra, ca, rb, cb, lda_d, ldb_d, ldc_d;
-  size_t off_b, off_c, total;
+  size_t off_b, off_c, off_cold, total;
+  bool by_k;  // k-chunks first
 };
+
+constexpr int64_t kChunkMinK = 2048;         // k-chunks pay from here on ...
+constexpr int64_t kChunkMinMN = 1ll << 22;   // ... for at least this many elements of C
+constexpr int kMaxChunks = 8;
 
 bool h_is_n(char c) { return c == 'N' || c == 'n'; }
 
@@ -31,7 +46,9 @@ HostPlan host_plan(int elem, char transa, char transb, int64_t m, int64_t n, int
   const size_t sa = round_up((size_t)p.lda_d * (size_t)(p.ca > 0 ? p.ca : 0) * elem, 256);
   const size_t sb = round_up((size_t)p.ldb_d * (size_t)(p.cb > 0 ? p.cb : 0) * elem, 256);
   const size_t sc = round_up((size_t)p.ldc_d * (size_t)(n > 0 ? n : 0) * elem, 256);
-  p.off_b = sa, p.off_c = sa + sb, p.total = sa + sb + sc;
+  p.by_k = k >= kChunkMinK && m * n >= kChunkMinMN;
+  p.off_b = sa, p.off_c = sa + sb, p.off_cold = sa + sb + sc;
+  p.total = sa + sb + sc + (p.by_k ? sc : 0);  // by k: the old values of C wait in a buffer of their own
   return p;
 }
 
@@ -39,8 +56,18 @@ HostPlan host_plan(int elem, char transa, char transb, int64_t m, int64_t n, int
 constexpr int kMaxPanels = 16;
 struct HostPipe {
   cudaStream_t cin, cout;
-  cudaEvent_t start, a_ready, out_done, in[kMaxPanels], done[kMaxPanels];
+  cudaEvent_t start, a_ready, out_done, in[kMaxPanels], done[kMaxPanels], old_in[kMaxPanels];
 };
+
+// C(:, 0:cols) += beta * Cold(:, 0:cols), both with leading dimension ld
+template <typename T>
+__global__ void add_scaled_kernel(int64_t rows, int64_t cols, T beta, T* C, const T* Cold, int64_t ld) {
+  const int64_t total = rows * cols;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t at = (i / rows) * ld + i % rows;
+    C[at] = C[at] + beta * Cold[at];
+  }
+}
 HostPipe* host_pipe() {
   static HostPipe pipes[64];
   static bool ready[64] = {};
@@ -52,7 +79,7 @@ HostPipe* host_pipe() {
                 cudaStreamCreateWithFlags(&h.cout, cudaStreamNonBlocking) == cudaSuccess;
     auto ev = [&good](cudaEvent_t* e) { good = good && cudaEventCreateWithFlags(e, cudaEventDisableTiming) == cudaSuccess; };
     ev(&h.start), ev(&h.a_ready), ev(&h.out_done);
-    for (int i = 0; i < kMaxPanels; ++i) ev(&h.in[i]), ev(&h.done[i]);
+    for (int i = 0; i < kMaxPanels; ++i) ev(&h.in[i]), ev(&h.done[i]), ev(&h.old_in[i]);
     if (!good) return nullptr;
     ready[dev] = true;
   }
@@ -92,6 +119,80 @@ int gemm_host(char transa, char transb, int64_t m, int64_t n, int64_t k, T alpha
   if (!ok(cudaEventRecord(hp->start, st)) || !ok(cudaStreamWaitEvent(hp->cin, hp->start, 0)) ||
       !ok(cudaStreamWaitEvent(hp->cout, hp->start, 0)))
     return B2_ERR_LAUNCH;
+  if (p.by_k && !scale_only) {
+    // ---- k-chunks first -------------------------------------------------------------------------------
+    const bool ta = !h_is_n(transa);
+    T* dCold = reinterpret_cast<T*>(w + p.off_cold);
+    int64_t chunks = k / 1024;
+    chunks = chunks < 2 ? 2 : (chunks > kMaxChunks ? kMaxChunks : chunks);
+    const int64_t kc = ((k + chunks - 1) / chunks + 63) / 64 * 64;
+    // The first chunks are added to all of C as they arrive; the last three eighths of k are applied column
+    // panel by column panel, so that finished panels leave over about as long as the copy back of C takes
+    // (a third of the multiplication on this machine) instead of all at the end.
+    const int64_t nchunks = (k + kc - 1) / kc;
+    int64_t late = (3 * nchunks + 4) / 8;
+    late = late < 1 ? 1 : late;
+    const int64_t k1 = (nchunks - late) * kc;  // first k of the part applied by panels
+    int nc = 0;
+    for (int64_t k0 = 0; k0 < k; k0 += kc, ++nc) {
+      const int64_t kk = (k - k0) < kc ? (k - k0) : kc;
+      // chunk of op(A): columns k0.. of an m x k matrix, or rows k0.. of a k x m one; of op(B) the other way round
+      cudaError_t err =
+          ta ? cudaMemcpy2DAsync(dA + k0, p.lda_d * e, A + k0, lda * e, kk * e, p.ca, cudaMemcpyHostToDevice, hp->cin)
+             : cudaMemcpy2DAsync(dA + k0 * p.lda_d, p.lda_d * e, A + k0 * lda, lda * e, p.ra * e, kk,
+                                 cudaMemcpyHostToDevice, hp->cin);
+      if (!ok(err)) return B2_ERR_LAUNCH;
+      err = tb ? cudaMemcpy2DAsync(dB + k0 * p.ldb_d, p.ldb_d * e, B + k0 * ldb, ldb * e, p.rb * e, kk,
+                                   cudaMemcpyHostToDevice, hp->cin)
+               : cudaMemcpy2DAsync(dB + k0, p.ldb_d * e, B + k0, ldb * e, kk * e, p.cb, cudaMemcpyHostToDevice, hp->cin);
+      if (!ok(err)) return B2_ERR_LAUNCH;
+      if (!ok(cudaEventRecord(hp->in[nc], hp->cin)) || !ok(cudaStreamWaitEvent(st, hp->in[nc], 0))) return B2_ERR_LAUNCH;
+      if (k0 < k1) {
+        const int rc = gemm_entry<T>(B2_VARIANT_AUTO, transa, transb, m, n, kk, alpha, ta ? dA + k0 : dA + k0 * p.lda_d,
+                                     p.lda_d, tb ? dB + k0 * p.ldb_d : dB + k0, p.ldb_d, k0 == 0 ? T(0) : T(1), dC,
+                                     p.ldc_d, cuda_stream);
+        if (rc) return rc;
+      }
+    }
+    // the old values of C follow A and B, panel by panel
+    int np = 0;
+    if (beta != T(0)) {
+      for (int64_t j0 = 0; j0 < n; j0 += width, ++np) {
+        const int64_t nj = (n - j0) < width ? (n - j0) : width;
+        if (!ok(cudaMemcpy2DAsync(dCold + j0 * p.ldc_d, p.ldc_d * e, C + j0 * ldc, ldc * e, m * e, nj,
+                                  cudaMemcpyHostToDevice, hp->cin)) ||
+            !ok(cudaEventRecord(hp->old_in[np], hp->cin)))
+          return B2_ERR_LAUNCH;
+      }
+    }
+    // the rest of k (all of A and B is on the device: the caller's stream has waited for every chunk)
+    const T* dAk = ta ? dA + k1 : dA + k1 * p.lda_d;
+    const T* dBk = tb ? dB + k1 * p.ldb_d : dB + k1;
+    np = 0;
+    for (int64_t j0 = 0; j0 < n; j0 += width, ++np) {
+      const int64_t nj = (n - j0) < width ? (n - j0) : width;
+      T* dCj = dC + j0 * p.ldc_d;
+      const int rc = gemm_entry<T>(B2_VARIANT_AUTO, transa, transb, m, nj, k - k1, alpha, dAk, p.lda_d,
+                                   tb ? dBk + j0 : dBk + j0 * p.ldb_d, p.ldb_d, k1 == 0 ? T(0) : T(1), dCj, p.ldc_d,
+                                   cuda_stream);
+      if (rc) return rc;
+      if (beta != T(0)) {
+        if (!ok(cudaStreamWaitEvent(st, hp->old_in[np], 0))) return B2_ERR_LAUNCH;
+        const int64_t blocks = (m * nj + 255) / 256, cap = (int64_t)sm_count_cached() * 16;
+        add_scaled_kernel<T><<<(unsigned)(blocks > cap ? cap : blocks), 256, 0, st>>>(m, nj, beta, dCj,
+                                                                                   dCold + j0 * p.ldc_d, p.ldc_d);
+        if (cudaGetLastError() != cudaSuccess) return B2_ERR_LAUNCH;
+      }
+      if (!ok(cudaEventRecord(hp->done[np], st)) || !ok(cudaStreamWaitEvent(hp->cout, hp->done[np], 0)) ||
+          !ok(cudaMemcpy2DAsync(C + j0 * ldc, ldc * e, dCj, p.ldc_d * e, m * e, nj, cudaMemcpyDeviceToHost, hp->cout)))
+        return B2_ERR_LAUNCH;
+    }
+    if (!ok(cudaEventRecord(hp->out_done, hp->cout)) || !ok(cudaStreamWaitEvent(st, hp->out_done, 0)))
+      return B2_ERR_LAUNCH;
+    return cudaStreamSynchronize(st) == cudaSuccess ? B2_OK : B2_ERR_LAUNCH;
+  }
+
+  // ---- column panels of C ---------------------------------------------------------------------------------
   if (!scale_only) {
     if (!ok(cudaMemcpy2DAsync(dA, p.lda_d * e, A, lda * e, p.ra * e, p.ca, cudaMemcpyHostToDevice, hp->cin)))
       return B2_ERR_LAUNCH;

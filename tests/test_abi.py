@@ -79,7 +79,9 @@ def test_workspace_sizes(b2):
     assert b2.b2_zgemm4m_workspace_bytes("X", "N", 3, 5, 7) == 0
     assert b2.b2_zgemm4m_workspace_bytes("C", "N", 3, 5, 7) == b2.b2_zgemm4m_workspace_bytes("T", "N", 3, 5, 7)
     assert b2.b2_zgemm3m_workspace_bytes("N", "N", 4096, 4096, 4096) == 9 * 4096 * 4096 * 8
-    assert b2.b2_gemm_host_workspace_bytes(0, "N", "N", 8192, 8192, 8192) == 3 * 8192 * 8192 * 8
+    # A, B, C, and for large problems a second buffer of C's size (the old values of C arrive last)
+    assert b2.b2_gemm_host_workspace_bytes(0, "N", "N", 8192, 8192, 8192) == 4 * 8192 * 8192 * 8
+    assert b2.b2_gemm_host_workspace_bytes(0, "N", "N", 1024, 1024, 1024) == 3 * 1024 * 1024 * 8
     assert b2.b2_gemm_host_workspace_bytes(1, "T", "N", 1001, 999, 1003) >= 4 * (1003 * 1001 + 1003 * 999 + 1001 * 999)
 
 

@@ -385,6 +385,44 @@ def test_host_entry_matches_oracle(b2, oracle, kind):
         assert np.all(err <= 2 * k * u * S.reshape(n, m))
 
 
+@pytest.mark.parametrize("kind", ["d", "s"])
+def test_host_entry_large_k_chunks(b2, oracle, kind):
+    """Large problems go up chunk by chunk along k and are accumulated as the chunks arrive (ragged last chunk and
+    last panel, padded leading dimensions, all transposes); the old values of C are added at the end from a buffer
+    of their own, and beta == 0 must not read C (NaN there).  Checked on a column sample: exact on integer data,
+    within the bound otherwise."""
+    tdt = torch.float64 if kind == "d" else torch.float32
+    fn = b2.b2_dgemm_host if kind == "d" else b2.b2_sgemm_host
+    u = 2.0 ** -53 if kind == "d" else 2.0 ** -24
+    m, n, k = 2100, 2050, 2250
+    assert b2.b2_gemm_host_workspace_bytes(0 if kind == "d" else 1, "N", "N", m, n, k) >= 4 * m * n * (8 if kind == "d" else 4)
+    cols = sample_columns(n, tile=64, extra=6, seed=5)
+    for ta, tb in TRANS:
+        (ra, ca), (rb, cb) = synth.operand_shapes(ta, tb, m, n, k)
+        for dist, alpha, beta in (("uniform", 0.7, -0.3), ("int9", 1.5, 0.5), ("int9", 1.0, 0.0)):
+            A, lda, B, ldb, C, ldc = synth.gemm_inputs(ta, tb, m, n, k, dist, 63, tdt, ra + 5, rb + 3, m + 7)
+            if beta == 0.0:
+                C.fill_(float("nan"))
+            want = C.numpy().copy()
+            oracle.ref_gemm(ta, tb, m, n, k, alpha, A.numpy(), lda, B.numpy(), ldb, beta, want, ldc, cols=cols)
+            ws = torch.empty(b2.b2_gemm_host_workspace_bytes(0 if kind == "d" else 1, ta, tb, m, n, k),
+                             dtype=torch.uint8, device="cuda")
+            Ch = C.clone().pin_memory()
+            fn(ta, tb, m, n, k, alpha, A.pin_memory(), lda, B.pin_memory(), ldb, beta, Ch, ldc, ws)
+            assert b2.b2_device_status() == 0
+            got = Ch.numpy().reshape(n, ldc)
+            assert got[:, m:].tobytes() == C.numpy().reshape(n, ldc)[:, m:].tobytes()  # padding rows untouched
+            g, w_ = got[cols][:, :m], want.reshape(n, ldc)[cols][:, :m]
+            if dist == "int9":
+                assert g.tobytes() == w_.tobytes()
+            else:
+                _, S = oracle.ref_gemm_hi(ta, tb, m, n, k, alpha, A.numpy(), lda, B.numpy(), ldb, beta, C.numpy(), ldc,
+                                          cols=cols)
+                err = np.abs(g.astype(np.float64) - w_.astype(np.float64))
+                assert np.all(err <= 2 * k * u * S.reshape(n, m)[cols])
+            del ws
+
+
 # ---- selector and probe ----------------------------------------------------------------------------
 
 def test_query_config_reports_launch(b2):
