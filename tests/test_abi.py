@@ -104,7 +104,12 @@ def test_selector_is_sane_without_gpu(b2):
         assert cfg["grid"] == cfg["tiles_m"] * cfg["tiles_n"] * cfg["k_split"]
     assert big["micro_kernel"] == "dmma_tma" and tiny["BM"] * tiny["BN"] <= 32 * 32
     f32 = json.loads(b2.b2_gemm_query_config(1, "N", "T", 4096, 4096, 4096, 4096, 4096, 4096))
-    assert f32["micro_kernel"] == "ffma2" and f32["dtype"] == "f32"
+    # NT with 16-byte aligned columns: the one case where the TMA-staged fp32 kernel is the measured best
+    assert f32["micro_kernel"] == "ffma2_tma" and f32["dtype"] == "f32"
+    f32 = json.loads(b2.b2_gemm_query_config(1, "N", "N", 4096, 4096, 4096, 4096, 4096, 4096))
+    assert f32["micro_kernel"] == "ffma2"
+    f32 = json.loads(b2.b2_gemm_query_config(1, "N", "T", 4096, 4096, 4096, 4097, 4096, 4096))
+    assert f32["micro_kernel"] == "ffma2"  # odd leading dimension: no tensor map
     with pytest.raises(b2.B2Error):
         b2.b2_gemm_query_config(0, "N", "N", 8, 8, 8, 4, 8, 8)
     with pytest.raises(b2.B2Error):
