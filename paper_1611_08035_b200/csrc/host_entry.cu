@@ -53,7 +53,7 @@ HostPlan host_plan(int elem, char transa, char transb, int64_t m, int64_t n, int
 }
 
 // Helper streams and events of the pipelined host-buffer calls, one set per device, created on first use.
-constexpr int kMaxPanels = 16;
+constexpr int kMaxPanels = 20;  // events per kind; the panel count itself is capped at 16 (+1 for a cut last panel)
 struct HostPipe {
   cudaStream_t cin, cout;
   cudaEvent_t start, a_ready, out_done, in[kMaxPanels], done[kMaxPanels], old_in[kMaxPanels];
@@ -111,7 +111,7 @@ int gemm_host(char transa, char transb, int64_t m, int64_t n, int64_t k, T alpha
 
   // column panels of C: at least 512 columns each, at most kMaxPanels, multiples of 64 columns
   int64_t panels = n / 1024;
-  panels = panels < 1 ? 1 : (panels > kMaxPanels ? kMaxPanels : panels);
+  panels = panels < 1 ? 1 : (panels > 16 ? 16 : panels);
   const int64_t width = ((n + panels - 1) / panels + 63) / 64 * 64;
   const bool tb = !h_is_n(transb);
 
@@ -133,9 +133,29 @@ int gemm_host(char transa, char transb, int64_t m, int64_t n, int64_t k, T alpha
     int64_t late = (3 * nchunks + 4) / 8;
     late = late < 1 ? 1 : late;
     const int64_t k1 = (nchunks - late) * kc;  // first k of the part applied by panels
-    int nc = 0;
-    for (int64_t k0 = 0; k0 < k; k0 += kc, ++nc) {
-      const int64_t kk = (k - k0) < kc ? (k - k0) : kc;
+    // chunk boundaries; the first chunk is cut once more, a quarter first, so that the multiplication starts sooner
+    int64_t kb[kMaxChunks + 3];
+    int nb = 0;
+    kb[nb++] = 0;
+    const int64_t quarter = kc / 4 / 64 * 64;
+    if (quarter >= 128) kb[nb++] = quarter;
+    for (int64_t k0 = kc; k0 < k; k0 += kc) kb[nb++] = k0;
+    kb[nb] = k;
+    // column panels of the last part; the last panel is cut in two, so that less is left to copy back at the end
+    int64_t jb[kMaxPanels + 1];
+    int npanels = 0;
+    for (int64_t j0 = 0; j0 < n; j0 += width) jb[npanels++] = j0;
+    jb[npanels] = n;
+    {
+      const int64_t last = n - jb[npanels - 1], half = last / 2 / 64 * 64;
+      if (half >= 128 && npanels < kMaxPanels) {
+        jb[npanels + 1] = n;
+        jb[npanels] = jb[npanels - 1] + half;
+        ++npanels;
+      }
+    }
+    for (int nc = 0; nc < nb; ++nc) {
+      const int64_t k0 = kb[nc], kk = kb[nc + 1] - k0;
       // chunk of op(A): columns k0.. of an m x k matrix, or rows k0.. of a k x m one; of op(B) the other way round
       cudaError_t err =
           ta ? cudaMemcpy2DAsync(dA + k0, p.lda_d * e, A + k0, lda * e, kk * e, p.ca, cudaMemcpyHostToDevice, hp->cin)
@@ -155,10 +175,9 @@ int gemm_host(char transa, char transb, int64_t m, int64_t n, int64_t k, T alpha
       }
     }
     // the old values of C follow A and B, panel by panel
-    int np = 0;
     if (beta != T(0)) {
-      for (int64_t j0 = 0; j0 < n; j0 += width, ++np) {
-        const int64_t nj = (n - j0) < width ? (n - j0) : width;
+      for (int np = 0; np < npanels; ++np) {
+        const int64_t j0 = jb[np], nj = jb[np + 1] - j0;
         if (!ok(cudaMemcpy2DAsync(dCold + j0 * p.ldc_d, p.ldc_d * e, C + j0 * ldc, ldc * e, m * e, nj,
                                   cudaMemcpyHostToDevice, hp->cin)) ||
             !ok(cudaEventRecord(hp->old_in[np], hp->cin)))
@@ -168,9 +187,8 @@ int gemm_host(char transa, char transb, int64_t m, int64_t n, int64_t k, T alpha
     // the rest of k (all of A and B is on the device: the caller's stream has waited for every chunk)
     const T* dAk = ta ? dA + k1 : dA + k1 * p.lda_d;
     const T* dBk = tb ? dB + k1 * p.ldb_d : dB + k1;
-    np = 0;
-    for (int64_t j0 = 0; j0 < n; j0 += width, ++np) {
-      const int64_t nj = (n - j0) < width ? (n - j0) : width;
+    for (int np = 0; np < npanels; ++np) {
+      const int64_t j0 = jb[np], nj = jb[np + 1] - j0;
       T* dCj = dC + j0 * p.ldc_d;
       const int rc = gemm_entry<T>(B2_VARIANT_AUTO, transa, transb, m, nj, k - k1, alpha, dAk, p.lda_d,
                                    tb ? dBk + j0 : dBk + j0 * p.ldb_d, p.ldb_d, k1 == 0 ? T(0) : T(1), dCj, p.ldc_d,
