@@ -148,8 +148,41 @@ static bool operands_aligned(const T* A, int64_t lda, const T* B, int64_t ldb) {
 // 2 / 4): 768^3 45.1 / 28.7 / 36.9, 1024^3 57.9 / 53.7 / 58.0, 1536^3 141 / 142 / 162, 2048^3 355 / 312 / 343,
 // 3072^3 1031 / 1031 / 1086.
 template <typename T>
+int choose_variant_uncached(int64_t m, int64_t n, int64_t k, bool aligned, int64_t batch, bool ta, bool tb,
+                            int* ksplit_out);
+
+// The choice is a pure function of its arguments (and of the device's SM count) that costs a few microseconds of
+// model arithmetic: as much as a small problem's kernel.  Each host thread remembers its last few choices.
+template <typename T>
 int choose_variant(int64_t m, int64_t n, int64_t k, bool aligned, int64_t batch = 1, bool ta = false,
                    bool tb = false, int* ksplit_out = nullptr) {
+  struct Entry {
+    int64_t m, n, k, batch;
+    int flags, sms, variant, ksplit;
+  };
+  constexpr int kEntries = 16;
+  thread_local Entry cache[kEntries] = {};
+  thread_local int next = 0;
+  const int flags = 1 | (aligned ? 2 : 0) | (ta ? 4 : 0) | (tb ? 8 : 0) | (ksplit_out ? 16 : 0);  // never 0
+  const int sms = sm_count_cached();
+  for (int i = 0; i < kEntries; ++i) {
+    const Entry& e = cache[i];
+    if (e.flags == flags && e.m == m && e.n == n && e.k == k && e.batch == batch && e.sms == sms) {
+      if (ksplit_out) *ksplit_out = e.ksplit;
+      return e.variant;
+    }
+  }
+  int ksplit = 1;
+  const int v = choose_variant_uncached<T>(m, n, k, aligned, batch, ta, tb, ksplit_out ? &ksplit : nullptr);
+  cache[next] = Entry{m, n, k, batch, flags, sms, v, ksplit};
+  next = (next + 1) % kEntries;
+  if (ksplit_out) *ksplit_out = ksplit;
+  return v;
+}
+
+template <typename T>
+int choose_variant_uncached(int64_t m, int64_t n, int64_t k, bool aligned, int64_t batch, bool ta, bool tb,
+                            int* ksplit_out) {
   const bool tma_ok = aligned && batch <= 1;
   const int count = variant_count_t<T>();
   TileChoice cand[16];
