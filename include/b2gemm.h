@@ -17,9 +17,10 @@
  *     (or from the first call that needs it) until the process exits, is: the scratch array of
  *     b2_zgemm4m_static (B2_ZGEMM4M_STATIC_BYTES of device memory on every GPU that loads the
  *     library), two device status words (b2_device_status), per-device caches of symbol
- *     addresses, shared-memory attributes and the SM count, and, for the host-buffer forms, two
- *     helper streams and a few events per device.  None of it carries results from one call to
- *     the next.
+ *     addresses, shared-memory attributes and the SM count, per host thread the last sixteen
+ *     kernel choices of the selector (a pure function of the problem's shape), and, for the
+ *     host-buffer forms, two helper streams and a few events per device.  None of it carries
+ *     results from one call to the next.
  *   - Threads: the per-device caches are filled on first use through atomic slots and one-time
  *     initialisers, so host threads may make their first calls concurrently.  Calls that share
  *     an output or a workspace must be ordered by the caller.
