@@ -183,7 +183,8 @@ int choose_variant(int64_t m, int64_t n, int64_t k, bool aligned, int64_t batch 
 template <typename T>
 int choose_variant_uncached(int64_t m, int64_t n, int64_t k, bool aligned, int64_t batch, bool ta, bool tb,
                             int* ksplit_out) {
-  const bool tma_ok = aligned && batch <= 1;
+  // tensor-map coordinates are 32-bit
+  const bool tma_ok = aligned && batch <= 1 && m <= 0x7fffffffLL && n <= 0x7fffffffLL && k <= 0x7fffffffLL;
   const int count = variant_count_t<T>();
   TileChoice cand[16];
   for (int v = 0; v < count && v < 16; ++v) {

@@ -108,6 +108,9 @@ def test_selector_is_sane_without_gpu(b2):
     assert f32["micro_kernel"] == "ffma2_tma" and f32["dtype"] == "f32"
     f32 = json.loads(b2.b2_gemm_query_config(1, "N", "N", 4096, 4096, 4096, 4096, 4096, 4096))
     assert f32["micro_kernel"] == "ffma2"
+    # tensor-map coordinates are 32-bit: an extent beyond that keeps the selector off the TMA-staged kernels
+    long_k = json.loads(b2.b2_gemm_query_config(0, "N", "N", 4096, 4096, 2 ** 31 + 64, 4096, 2 ** 31 + 64, 4096))
+    assert long_k["micro_kernel"] == "dmma"
     f32 = json.loads(b2.b2_gemm_query_config(1, "N", "T", 4096, 4096, 4096, 4097, 4096, 4096))
     assert f32["micro_kernel"] == "ffma2"  # odd leading dimension: no tensor map
     with pytest.raises(b2.B2Error):
