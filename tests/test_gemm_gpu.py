@@ -155,6 +155,16 @@ def test_tma_variants_aligned_ragged_shapes(b2, oracle, kind):
                 r = run_and_check(b2, oracle, kind, ta, tb, m, n, k, 1.5, 0.5, dist="int9", seed=m + k, variant=v,
                                   lds=lds, expect_exact=True)
                 assert r is not None
+            # beta == 1: interior tiles of the fp64 kernels leave by bulk reductions that add to C in memory, edge
+            # tiles and a C with an odd leading dimension by the ordinary epilogue -- both in one launch here
+            for (m, n, k) in [(200, 136, 75), (333, 270, 145)]:
+                (ra, _), (rb, _) = synth.operand_shapes(ta, tb, m, n, k)
+                for ldc in (m + (m & 1) + 2, m | 1):
+                    lds = ((ra + vec - 1) // vec * vec + vec, (rb + vec - 1) // vec * vec, ldc)
+                    assert run_and_check(b2, oracle, kind, ta, tb, m, n, k, -1.0, 1.0, seed=m + k + 1, variant=v,
+                                         lds=lds) is not None
+                    assert run_and_check(b2, oracle, kind, ta, tb, m, n, k, -1.0, 1.0, dist="int9", seed=m + k + 1,
+                                         variant=v, lds=lds, expect_exact=True) is not None
 
 
 def test_bounded_wait_reports_timeout(b2):
