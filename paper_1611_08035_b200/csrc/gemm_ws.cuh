@@ -223,8 +223,10 @@ struct GemmWsKernel {
     for (int i = g, u = 0; i < my_tiles && ok; i += GROUPS, ++u) {
       int m0, n0;
       tile_origin(i, m0, n0);
-      // beta != 0: pull the tile's old C values towards L2 while the k-loop runs
-      if (use_beta) {
+      // beta != 0: pull the tile's old C values towards L2 while the k-loop runs (not when the tile will be added
+      // to C in memory: nothing waits for those values then)
+      const bool will_add = STAGE_C && c_vec_ok && p.beta == T(1) && (int64_t)m0 + BM <= p.m && (int64_t)n0 + BN <= p.n;
+      if (use_beta && !will_add) {
         const int m_valid = (int)min((int64_t)BM, p.m - m0), n_valid = (int)min((int64_t)BN, p.n - n0);
         constexpr int LINE = 16, LPC = BM / LINE;  // 128-byte lines per tile column
         for (int c = ltid; c < BN * LPC; c += GT) {
@@ -261,7 +263,10 @@ struct GemmWsKernel {
       // ---- drain: fused alpha/beta epilogue ----
       // through the staging tile when the whole tile lies inside C and its columns are 16-byte aligned
       const bool staged = STAGE_C && c_vec_ok && (int64_t)m0 + BM <= p.m && (int64_t)n0 + BN <= p.n;
+      // beta == 1 on a staged tile: nothing of C is loaded; the tile is added to C in memory by bulk reductions
+      const bool add_in_memory = staged && p.beta == T(1);
       if (staged) {
+        const bool use_beta = p.beta != T(0) && !add_in_memory;
         T* cfrag = p.C + (int64_t)(n0 + fcol) * p.ldc + m0 + frow;
         // results into the accumulator registers; the old values are fetched in C_BATCHES batches
 #pragma unroll
@@ -322,7 +327,10 @@ struct GemmWsKernel {
               ok = false;
               break;
             }
-            bulk_store(p.C + (int64_t)(n0 + ltid) * p.ldc + m0, cbuf + ltid * C_PITCH, COL_BYTES);
+            if (add_in_memory)
+              bulk_reduce_add_f64(p.C + (int64_t)(n0 + ltid) * p.ldc + m0, cbuf + ltid * C_PITCH, COL_BYTES);
+            else
+              bulk_store(p.C + (int64_t)(n0 + ltid) * p.ldc + m0, cbuf + ltid * C_PITCH, COL_BYTES);
             bulk_commit();
             bulk_wait_read_all();  // the column has left the staging tile
           }
