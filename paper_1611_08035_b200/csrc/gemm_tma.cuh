@@ -194,8 +194,10 @@ struct GemmTmaKernel {
 
     // beta == 1 (C := C + alpha A B, the trailing update of a factorisation), interior tile, 16-byte aligned
     // columns of C, fp64 tensor-core micro-kernel: the tile will be ADDED to C in memory (see the drain below)
-    const bool by_reduction = sizeof(T) == 8 && p.beta == T(1) && p.tri == 0 && m0 + BM <= p.m && n0 + BN <= p.n &&
-                              (reinterpret_cast<uintptr_t>(p.C) & 15) == 0 && (p.ldc & 1) == 0;
+    // (in a triangular update: a tile that lies wholly inside the stored triangle)
+    const bool by_reduction = sizeof(T) == 8 && p.beta == T(1) && !tile_crosses_diagonal(p.tri, m0, n0, BM, BN) &&
+                              m0 + BM <= p.m && n0 + BN <= p.n && (reinterpret_cast<uintptr_t>(p.C) & 15) == 0 &&
+                              (p.ldc & 1) == 0;
 
     // beta != 0: pull the tile's old C values towards L2 while the k-loop runs (not for a tile that is added in
     // memory: no thread will wait for those values, and the update measures 2 % faster without the prefetch)
