@@ -176,6 +176,28 @@ struct SimtTmaMicro {
     }
   }
 
+  // alpha * acc into a column-major tile in shared memory (column pitch PC, 16-byte aligned columns)
+  static constexpr int PC = BM + 4;
+  static __device__ __forceinline__ void stage_tile(const Acc& acc, float alpha, float* sC, int warp_m, int warp_n,
+                                                    int lane) {
+    const int lx = lane & 7, ly = lane >> 3;
+#pragma unroll
+    for (int j = 0; j < TN; ++j) {
+      float* col = sC + (warp_n * WTN + col_of(j, ly)) * PC + warp_m * WTM;
+#pragma unroll
+      for (int g = 0; g < TM / 4; ++g) {
+        if constexpr (!A_KC) {  // four neighbouring rows
+          *reinterpret_cast<float4*>(col + row_of(4 * g, lx)) =
+              make_float4(alpha * get(acc, 4 * g, j), alpha * get(acc, 4 * g + 1, j), alpha * get(acc, 4 * g + 2, j),
+                          alpha * get(acc, 4 * g + 3, j));
+        } else {
+#pragma unroll
+          for (int e = 0; e < 4; ++e) col[row_of(4 * g + e, lx)] = alpha * get(acc, 4 * g + e, j);
+        }
+      }
+    }
+  }
+
   // C := alpha*acc + beta*C on the lane's block, column by column; rows >= m and columns >= n are skipped.
   static __device__ __forceinline__ void store(const Acc& acc, const GemmArgs<float>& p, float* C, int64_t m0,
                                                int64_t n0, int warp_m, int warp_n, int lane) {

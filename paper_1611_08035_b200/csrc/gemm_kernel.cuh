@@ -219,6 +219,22 @@ struct DmmaMicro {
     c = __dadd_rn(c, __longlong_as_double((long long)bits));
   }
 
+  // alpha * acc into a column-major tile in shared memory (column pitch PC, 16-byte aligned columns)
+  static constexpr int PC = BM + 2;
+  static __device__ __forceinline__ void stage_tile(const Acc& acc, double alpha, double* sC, int warp_m, int warp_n,
+                                                    int lane) {
+    const int g = lane >> 2, t = lane & 3;
+    const int r0 = warp_m * WTM + 2 * g, c0 = warp_n * WTN + 2 * t;
+#pragma unroll
+    for (int mi = 0; mi < MI; ++mi)
+#pragma unroll
+      for (int ni = 0; ni < NI; ++ni)
+#pragma unroll
+        for (int h = 0; h < 2; ++h)
+          *reinterpret_cast<double2*>(sC + (c0 + ni * 8 + h) * PC + r0 + mi * 16) =
+              make_double2(alpha * acc.c[mi][ni][h], alpha * acc.c[mi][ni][2 + h]);
+  }
+
   // sum of a lane's accumulators (probes keep their result alive through it)
   static __device__ __forceinline__ double checksum(const Acc& acc) {
     double s = 0.0;
@@ -598,6 +614,39 @@ struct SimtMicro {
 //   aligned, leading dimensions multiples of 16/sizeof(T)); otherwise operands are staged
 //   element by element.
 // ---------------------------------------------------------------------------------------
+// ---------------------------------------------------------------------------------------
+// Drain by reductions in memory, for beta == 1 (C := C + alpha op(A) op(B), the trailing update of a factorisation).
+// A tile that lies wholly inside C (and inside the stored triangle of a triangular update) and whose columns of C
+// are 16-byte aligned leaves as alpha * acc through shared memory that the operand ring no longer needs, and one
+// thread per column issues a bulk reduction that ADDS the column to C in memory.  No thread loads an old value of
+// C or waits for one.  The arithmetic is the ordinary epilogue's with beta = 1 (alpha * acc rounded, then one
+// addition to the old value), so the bits are the same.  Used by the TMA-staged kernels; in the cp.async fp32
+// kernels it was measured and changed nothing (16384^2 x 64: 42.9 against 43.4 TFLOP/s; their drain is not what
+// they wait for), and the cp.async fp64 64 x 64 kernel has no register to spare for it.
+// ---------------------------------------------------------------------------------------
+template <class Micro>
+__device__ __forceinline__ bool tile_added_in_memory(const GemmArgs<typename Micro::T>& p, const typename Micro::T* C,
+                                                     int64_t m0, int64_t n0) {
+  using T = typename Micro::T;
+  return p.beta == T(1) && !tile_crosses_diagonal(p.tri, m0, n0, Micro::BM, Micro::BN) && m0 + Micro::BM <= p.m &&
+         n0 + Micro::BN <= p.n && (reinterpret_cast<uintptr_t>(C) & 15) == 0 && (p.ldc % (16 / (int)sizeof(T))) == 0;
+}
+// Every thread of the CTA calls this after its last read of the ring; sC is the ring's first byte.
+template <class Micro>
+__device__ __forceinline__ void drain_by_reduction(const typename Micro::Acc& acc, const GemmArgs<typename Micro::T>& p,
+                                                   typename Micro::T* C, int64_t m0, int64_t n0,
+                                                   typename Micro::T* sC, int warp_m, int warp_n, int lane) {
+  using T = typename Micro::T;
+  __syncthreads();  // every warp has finished reading the ring
+  Micro::stage_tile(acc, p.alpha, sC, warp_m, warp_n, lane);
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // these writes are read by the async proxy
+  __syncthreads();
+  for (int c = threadIdx.x; c < Micro::BN; c += Micro::NT)
+    bulk_reduce_add(C + (n0 + c) * p.ldc + m0, sC + c * Micro::PC, (uint32_t)(Micro::BM * sizeof(T)));
+  bulk_commit();
+  bulk_wait_read_all();  // the shared memory must outlive the reads of the reductions
+}
+
 template <class Micro, int STAGES, bool TA, bool TB, bool ALIGNED>
 struct GemmKernel {
   using T = typename Micro::T;

@@ -104,16 +104,7 @@ __device__ __forceinline__ void bulk_store(void* gmem_dst, const void* smem_src,
                "r"(bytes)
                : "memory");
 }
-// shared -> global with an addition at the destination: every fp64 element of the block is ADDED to the element
-// in global memory (one IEEE addition each, done by the memory system); tracked like a bulk store
-__device__ __forceinline__ void bulk_reduce_add_f64(void* gmem_dst, const void* smem_src, uint32_t bytes) {
-  asm volatile("cp.reduce.async.bulk.global.shared::cta.bulk_group.add.f64 [%0], [%1], %2;" ::"l"(gmem_dst),
-               "r"(smem_u32(smem_src)), "r"(bytes)
-               : "memory");
-}
-__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-// all of this thread's bulk stores have read their shared-memory source / have completed
-__device__ __forceinline__ void bulk_wait_read_all() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+// all of this thread's bulk stores have completed (bulk_wait_read_all: have read their source)
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
 // ---- host helpers shared by the TMA-staged kernels (defined in gemm_f64_tma.cu) ------------------
@@ -192,12 +183,10 @@ struct GemmTmaKernel {
       for (; issued < STAGES - LAG && issued < KT; ++issued) issue(issued);
     }
 
-    // beta == 1 (C := C + alpha A B, the trailing update of a factorisation), interior tile, 16-byte aligned
-    // columns of C, fp64 tensor-core micro-kernel: the tile will be ADDED to C in memory (see the drain below)
-    // (in a triangular update: a tile that lies wholly inside the stored triangle)
-    const bool by_reduction = sizeof(T) == 8 && p.beta == T(1) && !tile_crosses_diagonal(p.tri, m0, n0, BM, BN) &&
-                              m0 + BM <= p.m && n0 + BN <= p.n && (reinterpret_cast<uintptr_t>(p.C) & 15) == 0 &&
-                              (p.ldc & 1) == 0;
+    // beta == 1, interior tile, 16-byte aligned columns of C: the tile will be ADDED to C in memory
+    // (drain_by_reduction in gemm_kernel.cuh)
+    constexpr bool REDUCE_OK = (size_t)STAGES * (A_BYTES + B_BYTES) >= (size_t)Micro::BN * Micro::PC * sizeof(T);
+    const bool by_reduction = REDUCE_OK && tile_added_in_memory<Micro>(p, p.C, m0, n0);
 
     // beta != 0: pull the tile's old C values towards L2 while the k-loop runs (not for a tile that is added in
     // memory: no thread will wait for those values, and the update measures 2 % faster without the prefetch)
@@ -258,31 +247,9 @@ struct GemmTmaKernel {
       }
       return;
     }
-    if constexpr (sizeof(T) == 8) {  // the fp64 tensor-core micro-kernels (fragment layout below)
-      // The tile leaves as alpha * acc through the idle ring and is ADDED to C in memory by bulk reductions, one
-      // per column.  No thread loads an old value of C or waits for one; the arithmetic is the same (alpha * acc
-      // rounded, then one addition to the old value), so are the bits.
-      constexpr int PC = BM + 2;  // column pitch in the ring: 16-byte aligned columns
-      static_assert((size_t)BN * PC * 8 <= (size_t)STAGES * (A_BYTES + B_BYTES), "the ring holds a tile of C");
+    if constexpr (REDUCE_OK) {
       if (by_reduction) {
-        __syncthreads();  // every warp has finished reading the ring
-        double* sC = reinterpret_cast<double*>(smem_raw);
-        const int g = lane >> 2, t = lane & 3;
-        const int r0 = warp_m * Micro::WTM + 2 * g, c0 = warp_n * Micro::WTN + 2 * t;
-#pragma unroll
-        for (int mi = 0; mi < Micro::MI; ++mi)
-#pragma unroll
-          for (int ni = 0; ni < Micro::NI; ++ni)
-#pragma unroll
-            for (int h = 0; h < 2; ++h)
-              *reinterpret_cast<double2*>(sC + (c0 + ni * 8 + h) * PC + r0 + mi * 16) =
-                  make_double2(p.alpha * acc.c[mi][ni][h], p.alpha * acc.c[mi][ni][2 + h]);
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // these writes are read by the async proxy
-        __syncthreads();
-        for (int c = tid; c < BN; c += NT)
-          bulk_reduce_add_f64(p.C + (n0 + c) * p.ldc + m0, sC + c * PC, (uint32_t)(BM * 8));
-        bulk_commit();
-        bulk_wait_read_all();  // the ring must outlive the reads of the reductions
+        drain_by_reduction<Micro>(acc, p, p.C, m0, n0, reinterpret_cast<T*>(smem_raw), warp_m, warp_n, lane);
         return;
       }
     }

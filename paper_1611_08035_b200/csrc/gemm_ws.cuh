@@ -328,7 +328,7 @@ struct GemmWsKernel {
               break;
             }
             if (add_in_memory)
-              bulk_reduce_add_f64(p.C + (int64_t)(n0 + ltid) * p.ldc + m0, cbuf + ltid * C_PITCH, COL_BYTES);
+              bulk_reduce_add(p.C + (int64_t)(n0 + ltid) * p.ldc + m0, cbuf + ltid * C_PITCH, COL_BYTES);
             else
               bulk_store(p.C + (int64_t)(n0 + ltid) * p.ldc + m0, cbuf + ltid * C_PITCH, COL_BYTES);
             bulk_commit();

@@ -132,6 +132,11 @@ def test_all_variants_multi_tile_ragged(b2, oracle, kind):
             run_and_check(b2, oracle, kind, ta, tb, 300, 260, 136, 1.0, 0.0, seed=v, pad=False, variant=v)
             run_and_check(b2, oracle, kind, ta, tb, 300, 260, 136, 1.5, 0.5, dist="int9", seed=v, variant=v,
                           expect_exact=True)
+            # beta == 1 with 16-byte aligned columns of C: interior tiles may be added to C in memory by bulk
+            # reductions (fp32 kernels, TMA-staged fp64 kernels), edge tiles take the ordinary epilogue
+            run_and_check(b2, oracle, kind, ta, tb, 300, 260, 136, -1.0, 1.0, seed=v + 1, variant=v)
+            run_and_check(b2, oracle, kind, ta, tb, 300, 260, 136, -1.0, 1.0, dist="int9", seed=v + 1, variant=v,
+                          expect_exact=True)
 
 
 @pytest.mark.parametrize("kind", ["d", "s"])
