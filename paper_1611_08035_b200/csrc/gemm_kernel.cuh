@@ -615,12 +615,13 @@ struct SimtMicro {
 //   element by element.
 // ---------------------------------------------------------------------------------------
 // ---------------------------------------------------------------------------------------
-// Drain by reductions in memory, for beta == 1 (C := C + alpha op(A) op(B), the trailing update of a factorisation).
-// A tile that lies wholly inside C (and inside the stored triangle of a triangular update) and whose columns of C
-// are 16-byte aligned leaves as alpha * acc through shared memory that the operand ring no longer needs, and one
-// thread per column issues a bulk reduction that ADDS the column to C in memory.  No thread loads an old value of
-// C or waits for one.  The arithmetic is the ordinary epilogue's with beta = 1 (alpha * acc rounded, then one
-// addition to the old value), so the bits are the same.  Used by the TMA-staged kernels; in the cp.async fp32
+// Drain through shared memory, for beta == 1 (C := C + alpha op(A) op(B), the trailing update of a factorisation)
+// and beta == 0.  A tile that lies wholly inside C (and inside the stored triangle of a triangular update) and
+// whose columns of C are 16-byte aligned leaves as alpha * acc through shared memory that the operand ring no
+// longer needs, and one thread per column issues a bulk copy: a reduction that ADDS the column to C in memory
+// (beta == 1), or a plain store (beta == 0).  No thread loads an old value of C, waits for one, or holds its
+// accumulators while stores drain.  The arithmetic is the ordinary epilogue's (alpha * acc rounded; with beta = 1
+// one addition to the old value), so the bits are the same.  Used by the TMA-staged kernels; in the cp.async fp32
 // kernels it was measured and changed nothing (16384^2 x 64: 42.9 against 43.4 TFLOP/s; their drain is not what
 // they wait for), and the cp.async fp64 64 x 64 kernel has no register to spare for it.
 // ---------------------------------------------------------------------------------------
@@ -628,7 +629,7 @@ template <class Micro>
 __device__ __forceinline__ bool tile_added_in_memory(const GemmArgs<typename Micro::T>& p, const typename Micro::T* C,
                                                      int64_t m0, int64_t n0) {
   using T = typename Micro::T;
-  return p.beta == T(1) && !tile_crosses_diagonal(p.tri, m0, n0, Micro::BM, Micro::BN) && m0 + Micro::BM <= p.m &&
+  return (p.beta == T(1) || p.beta == T(0)) && !tile_crosses_diagonal(p.tri, m0, n0, Micro::BM, Micro::BN) && m0 + Micro::BM <= p.m &&
          n0 + Micro::BN <= p.n && (reinterpret_cast<uintptr_t>(C) & 15) == 0 && (p.ldc % (16 / (int)sizeof(T))) == 0;
 }
 // Every thread of the CTA calls this after its last read of the ring; sC is the ring's first byte.
@@ -641,8 +642,12 @@ __device__ __forceinline__ void drain_by_reduction(const typename Micro::Acc& ac
   Micro::stage_tile(acc, p.alpha, sC, warp_m, warp_n, lane);
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // these writes are read by the async proxy
   __syncthreads();
-  for (int c = threadIdx.x; c < Micro::BN; c += Micro::NT)
-    bulk_reduce_add(C + (n0 + c) * p.ldc + m0, sC + c * Micro::PC, (uint32_t)(Micro::BM * sizeof(T)));
+  for (int c = threadIdx.x; c < Micro::BN; c += Micro::NT) {
+    if (p.beta == T(0))  // nothing to add to: a plain bulk store
+      bulk_store(C + (n0 + c) * p.ldc + m0, sC + c * Micro::PC, (uint32_t)(Micro::BM * sizeof(T)));
+    else
+      bulk_reduce_add(C + (n0 + c) * p.ldc + m0, sC + c * Micro::PC, (uint32_t)(Micro::BM * sizeof(T)));
+  }
   bulk_commit();
   bulk_wait_read_all();  // the shared memory must outlive the reads of the reductions
 }

@@ -98,12 +98,6 @@ __device__ __forceinline__ void bulk_load(void* smem_dst, const void* gmem_src, 
                "l"(gmem_src), "r"(bytes), "r"(smem_u32(bar))
                : "memory");
 }
-// shared -> global, tracked by the issuing thread's bulk async-groups
-__device__ __forceinline__ void bulk_store(void* gmem_dst, const void* smem_src, uint32_t bytes) {
-  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gmem_dst), "r"(smem_u32(smem_src)),
-               "r"(bytes)
-               : "memory");
-}
 // all of this thread's bulk stores have completed (bulk_wait_read_all: have read their source)
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
@@ -183,8 +177,8 @@ struct GemmTmaKernel {
       for (; issued < STAGES - LAG && issued < KT; ++issued) issue(issued);
     }
 
-    // beta == 1, interior tile, 16-byte aligned columns of C: the tile will be ADDED to C in memory
-    // (drain_by_reduction in gemm_kernel.cuh)
+    // beta == 1 or 0, interior tile, 16-byte aligned columns of C: the tile will leave through shared memory and be
+    // ADDED to C in memory, or stored, by bulk copies (drain_by_reduction in gemm_kernel.cuh)
     constexpr bool REDUCE_OK = (size_t)STAGES * (A_BYTES + B_BYTES) >= (size_t)Micro::BN * Micro::PC * sizeof(T);
     const bool by_reduction = REDUCE_OK && tile_added_in_memory<Micro>(p, p.C, m0, n0);
 
