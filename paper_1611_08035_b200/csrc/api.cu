@@ -149,13 +149,13 @@ static bool operands_aligned(const T* A, int64_t lda, const T* B, int64_t ldb) {
 // 3072^3 1031 / 1031 / 1086.
 template <typename T>
 int choose_variant_uncached(int64_t m, int64_t n, int64_t k, bool aligned, int64_t batch, bool ta, bool tb,
-                            int* ksplit_out);
+                            int* ksplit_out, bool drain_free);
 
 // The choice is a pure function of its arguments (and of the device's SM count) that costs a few microseconds of
 // model arithmetic: as much as a small problem's kernel.  Each host thread remembers its last few choices.
 template <typename T>
 int choose_variant(int64_t m, int64_t n, int64_t k, bool aligned, int64_t batch = 1, bool ta = false,
-                   bool tb = false, int* ksplit_out = nullptr) {
+                   bool tb = false, int* ksplit_out = nullptr, bool drain_free = false) {
   struct Entry {
     int64_t m, n, k, batch;
     int flags, sms, variant, ksplit;
@@ -163,7 +163,8 @@ int choose_variant(int64_t m, int64_t n, int64_t k, bool aligned, int64_t batch 
   constexpr int kEntries = 16;
   thread_local Entry cache[kEntries] = {};
   thread_local int next = 0;
-  const int flags = 1 | (aligned ? 2 : 0) | (ta ? 4 : 0) | (tb ? 8 : 0) | (ksplit_out ? 16 : 0);  // never 0
+  const int flags = 1 | (aligned ? 2 : 0) | (ta ? 4 : 0) | (tb ? 8 : 0) | (ksplit_out ? 16 : 0) |
+                    (drain_free ? 32 : 0);  // never 0
   const int sms = sm_count_cached();
   for (int i = 0; i < kEntries; ++i) {
     const Entry& e = cache[i];
@@ -173,7 +174,7 @@ int choose_variant(int64_t m, int64_t n, int64_t k, bool aligned, int64_t batch 
     }
   }
   int ksplit = 1;
-  const int v = choose_variant_uncached<T>(m, n, k, aligned, batch, ta, tb, ksplit_out ? &ksplit : nullptr);
+  const int v = choose_variant_uncached<T>(m, n, k, aligned, batch, ta, tb, ksplit_out ? &ksplit : nullptr, drain_free);
   cache[next] = Entry{m, n, k, batch, flags, sms, v, ksplit};
   next = (next + 1) % kEntries;
   if (ksplit_out) *ksplit_out = ksplit;
@@ -182,7 +183,7 @@ int choose_variant(int64_t m, int64_t n, int64_t k, bool aligned, int64_t batch 
 
 template <typename T>
 int choose_variant_uncached(int64_t m, int64_t n, int64_t k, bool aligned, int64_t batch, bool ta, bool tb,
-                            int* ksplit_out) {
+                            int* ksplit_out, bool drain_free) {
   // tensor-map coordinates are 32-bit
   const bool tma_ok = aligned && batch <= 1 && m <= 0x7fffffffLL && n <= 0x7fffffffLL && k <= 0x7fffffffLL;
   const int count = variant_count_t<T>();
@@ -197,7 +198,11 @@ int choose_variant_uncached(int64_t m, int64_t n, int64_t k, bool aligned, int64
     // transposed: no transposition anywhere), and serves plain single problems only (ksplit_out is null for
     // triangular updates)
     const bool fp32_tma = strcmp(vi.micro, "ffma2_tma") == 0;
-    const bool fp32_tma_fits = !ta && tb && ksplit_out != nullptr;
+    // ... and, for updates of up to 1024 in k whose tiles leave through shared memory (drain_free: beta is 0 or 1
+    // and the columns of C are 16-byte aligned), in NN and TT as well: measured at 2048^2 to 16384^2 with k = 64 to
+    // 2048, e.g. 16384^2 x 64, beta = 1: 51.0 against 43.1 TFLOP/s, x 256: 57.5 against 54.8, x 1024: 59.2 against 58.8
+    const bool short_update = drain_free && k <= 1024 && !(ta && !tb);
+    const bool fp32_tma_fits = ((!ta && tb) || short_update) && ksplit_out != nullptr;
     const bool needs_alignment = strcmp(vi.micro, "dmma_tma") == 0 || strcmp(vi.micro, "ffma2_tma") == 0;
     // Steady-state fraction of the arithmetic pipe at full residency: the pipeline model's prediction (Section 4
     // estimate x latency coverage x barrier stall, queue_model.h).  The table's measured value is the recorded check
@@ -214,7 +219,7 @@ int choose_variant_uncached(int64_t m, int64_t n, int64_t k, bool aligned, int64
     // Measured at 8192^3 (128 x 64 tile, TFLOP/s): NT 62.0, NN 59.2, TT 51.3, TN 47.1; 128 x 128: 63.7, 58.2, 56.8, 54.9.
     // The cost of B's copy differs per variant (128 x 64 transposes it through registers).
     if (fp32_tma) {
-      eff = 0.868;  // measured in NT at 8192^3 (the table's figure is NN, like the other fp32 rows)
+      eff = (!ta && tb) ? 0.868 : 0.86;  // NT at 8192^3; the short updates are set above the cp.async kernels
     } else if (strncmp(vi.micro, "ffma", 4) == 0 && sizeof(T) == 4) {
       const double ca = 10.0, cb = vi.transpose_b_cost;  // fitted to the eight figures above (within 4 %)
       double f = (1.0 - (ta ? ca / vi.bn : 0.0) - (tb ? 0.0 : cb / vi.bm)) / (1.0 - cb / vi.bm);
@@ -229,6 +234,21 @@ int choose_variant_uncached(int64_t m, int64_t n, int64_t k, bool aligned, int64
   }
   const int sms = sm_count_cached();
   int best = select_tile(cand, count < 16 ? count : 16, m, n, k, sms, (int)sizeof(T), batch);
+  // fp32 updates of up to 1024 in k whose tiles leave through shared memory, at least one and a half tiles of
+  // 128 x 128 per SM: the TMA-staged kernel is the measured best by 5 to 20 % in NN, NT and TT, which the estimate,
+  // fitted to kernels with the ordinary epilogue, does not see (2048^2 x 128: 35.5 against 31.6 TFLOP/s; below
+  // that tile count it loses: 1024^2 x 256 16.7 against 24.5)
+  if (sizeof(T) == 4 && drain_free && k <= 1024 && !(ta && !tb) && tma_ok && batch <= 1 && ksplit_out != nullptr) {
+    for (int v = 0; v < count && v < 16; ++v) {
+      const VariantInfo& vi = variant_info_t<T>(v);
+      if (strcmp(vi.micro, "ffma2_tma") != 0) continue;
+      const int64_t tiles = ((m + vi.bm - 1) / vi.bm) * ((n + vi.bn - 1) / vi.bn);
+      if (2 * tiles >= 3 * (int64_t)sms) {
+        *ksplit_out = 1;
+        return v;
+      }
+    }
+  }
   if (ksplit_out) {
     *ksplit_out = 1;
     double best_t = estimate_clks(cand[best], m, n, k, sms, (int)sizeof(T), batch);
@@ -271,7 +291,9 @@ int gemm_launch_checked(int variant, bool ta, bool tb, int64_t m, int64_t n, int
                        (ex.batch <= 1 || (ex.stride_a % kVec == 0 && ex.stride_b % kVec == 0));
   int ksplit = ex.ksplit > 0 ? ex.ksplit : 1;
   if (variant == B2_VARIANT_AUTO)
-    variant = choose_variant<T>(m, n, k, aligned, ex.batch, ta, tb, ex.tri == 0 ? &ksplit : nullptr);
+    variant = choose_variant<T>(m, n, k, aligned, ex.batch, ta, tb, ex.tri == 0 ? &ksplit : nullptr,
+                                (beta == T(0) || beta == T(1)) && (reinterpret_cast<uintptr_t>(C) & 15) == 0 &&
+                                    ldc % kVec == 0);
   GemmArgs<T> args;
   args.m = m, args.n = n, args.k = k;
   args.alpha = alpha, args.beta = beta;

@@ -117,6 +117,30 @@ def test_fp32_every_fma_variant_same_bits_8192(b2, oracle):
     _oracle_sample(oracle, "N", "N", m, n, k, 1.5, 0.5, A, lda, B, ldb, C, ldc, first, seed=13, extra=4)
 
 
+@pytest.mark.parametrize("ta,tb", [("N", "N"), ("T", "T"), ("N", "T")])
+def test_fp32_short_update_added_in_memory_8192(b2, oracle, ta, tb):
+    """C := C - op(A) op(B) on 8192^2 with k = 128 in fp32: the automatic choice is the TMA-staged kernel, whose
+    tiles are added to C in memory by bulk reductions (beta = 1) or leave by bulk stores (beta = 0); the cp.async
+    kernel with the ordinary epilogue must give the same bits over the whole matrix."""
+    m = n = 8192
+    k = 128
+    A, lda, B, ldb, C, ldc = synth.gemm_inputs(ta, tb, m, n, k, "int9", 2800, torch.float32, device="cuda")
+    for beta in (1.0, 0.0):
+        ref = C.clone()
+        b2.b2_sgemm(ta, tb, m, n, k, -1.0, A, lda, B, ldb, beta, ref, ldc, variant=1)
+        for rep in range(2):
+            got = C.clone()
+            b2.b2_sgemm(ta, tb, m, n, k, -1.0, A, lda, B, ldb, beta, got, ldc)
+            assert b2.b2_device_status() == 0
+            _assert_same(got, ref, f"automatic choice, beta {beta}, launch {rep}")
+        tma = [v for v in range(b2.b2_variant_count(1)) if staged_by_tma(b2.b2_variant_name(1, v))][0]
+        got = C.clone()
+        b2.b2_sgemm(ta, tb, m, n, k, -1.0, A, lda, B, ldb, beta, got, ldc, variant=tma)
+        _assert_same(got, ref, f"TMA-staged kernel, beta {beta}")
+        if beta == 1.0:
+            _oracle_sample(oracle, ta, tb, m, n, k, -1.0, 1.0, A, lda, B, ldb, C, ldc, ref, seed=19, extra=4)
+
+
 @pytest.mark.parametrize("size", [4096, 8192])
 def test_tf32_entries_against_the_fma_kernel_on_integer_data(b2, size):
     """Integers in {-4..4} are TF32 values and their sums stay below 2^24, so the one- and three-term tensor-core
