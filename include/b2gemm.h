@@ -128,7 +128,9 @@ const char* b2_variant_name(int dtype, int variant);
  * thread-block cluster the k-loop of each tile is divided, 1 = not divided; "grid" counts all CTAs) into
  * json_out (HOST memory, capacity cap bytes).  Returns 0, a negative argument index as above (dtype is
  * argument 1 here, the rest shift by one), or B2_ERR_WORKSPACE when cap is too small.
- * Nothing is launched.  The tile derivation follows the paper's register-limit formula
+ * Nothing is launched.  The answer is the one for a beta other than 0 and 1; with beta 0 or 1 and
+ * 16-byte aligned columns of C an fp32 update with k <= 1024 on enough tiles goes to the TMA-staged
+ * kernel instead (its tiles then leave through shared memory).  The tile derivation follows the paper's register-limit formula
  * (Section 5, "Limits imposed by registers") and pipeline-throughput estimate (Section 4).
  */
 int b2_gemm_query_config(int dtype, char transa, char transb, int64_t m, int64_t n, int64_t k, int64_t lda,
