@@ -266,6 +266,12 @@ def other_configs(b2, device, with_oracle=True):
         g = t["gflops"]
         peak = FP64_PEAK_TFLOPS if kind == "d" else FP32_PEAK_TFLOPS
         cfg = json.loads(b2.b2_gemm_query_config(0 if kind == "d" else 1, ta, tb, m, n, k, lda, ldb, ldc))
+        if kind == "s" and beta in (0.0, 1.0) and k <= 1024 and not pad and (ta, tb) != ("T", "N") \
+                and 2 * (-(-m // 128)) * (-(-n // 128)) >= 3 * torch.cuda.get_device_properties(device).multi_processor_count:
+            # the query answers for a general beta; such an update goes to the TMA-staged kernel (b2gemm.h)
+            cfg["name"] = [b2.b2_variant_name(1, v) for v in range(b2.b2_variant_count(1))
+                           if "tma" in b2.b2_variant_name(1, v)][0]
+            cfg["k_split"] = 1
         row = {"workload": label, "gflops": g, "gflops_best": t["gflops_best"], "ms_median": t["ms_median"],
                "launches": t["launches"], "frac_of_peak": round(g / 1e3 / peak, 4),
                "kernel": cfg["name"] + (f"/k_split {cfg['k_split']}" if cfg["k_split"] > 1 else "")}
@@ -277,7 +283,7 @@ def other_configs(b2, device, with_oracle=True):
             row["frac_of_peak_graph_replay"] = round(gg / 1e3 / peak, 4)
         if label.startswith("rank_k"):
             ms = 2.0 * m * n * k / g / 1e6
-            row["hbm_gbs"] = round((2.0 * m * n + (m + n) * k) * 8 / (ms * 1e-3) / 1e9, 1)
+            row["hbm_gbs"] = round((2.0 * m * n + (m + n) * k) * (8 if kind == "d" else 4) / (ms * 1e-3) / 1e9, 1)
         out.append(row)
         del A, B, C
 
@@ -292,6 +298,7 @@ def other_configs(b2, device, with_oracle=True):
                  f"{kind}gemm_{ta.lower()}{tb.lower()}_4096")
     for k in (64, 128, 256):
         real("d", "N", "N", 16384, 16384, k, -1.0, 1.0, "normal", 3000 + k, False, f"rank_k_dgemm_16384_k{k}")
+    real("s", "N", "N", 16384, 16384, 64, -1.0, 1.0, "normal", 3100, False, "rank_k_sgemm_16384_k64")
     for kind in "ds":
         for ta in "NT":
             for tb in "NT":
